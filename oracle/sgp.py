@@ -1,0 +1,139 @@
+"""Float64 oracle of the SGP / momentum-SGP / overlap-SGP recursion (test infrastructure).
+
+Written from Alg. 1 (SGP), Alg. 3 (SGP with Nesterov momentum) and Alg. 2
+(Overlap SGP) read through the supplementary delay model (virtual nodes, block
+mixing matrix, Eq. 4).  State is stacked by node: ``x`` is ``n x d`` (push-sum
+numerators), ``w`` is ``n`` (push-sum weights), ``u`` is ``n x d`` (momentum,
+never gossiped), ``z = x / w`` (de-biased parameters).
+
+Everything is float64 numpy, one statement per line of the algorithms, dense
+``P @ h`` for the mix.  No blocking, no fusion, nothing shared with the CUDA
+path.  Only tests, the smoke check and the benchmark's CPU-baseline leg may
+import this module.
+
+Readings fixed here where the paper leaves a choice:
+  * K steps means k = 0 .. K-1; u^(0) = 0; w^(0) = 1; z^(0) = x^(0).
+  * Weight decay adds lambda * x (the biased numerator the optimiser steps on,
+    App. C description of the compute thread) to the gradient.
+  * Delay tau: the self term p_ii h_i is never delayed; every other message
+    (p_ij h_j, p_ij w_j) sent at step k is added at step k + tau, i.e. it lands
+    in x^(k+tau+1); messages are sent every step; both parts accumulate;
+    virtual nodes start at zero.  For tau = 1 this is Alg. 2 ("always received
+    with 1 iteration of staleness", Table 4 caption).
+
+Pins: tests/test_oracle_sgp.py.
+"""
+from __future__ import annotations
+
+from collections import deque
+from dataclasses import dataclass, field
+
+import numpy as np
+
+
+@dataclass
+class SGPState:
+    x: np.ndarray                      # n x d numerators
+    w: np.ndarray                      # n push-sum weights
+    u: np.ndarray                      # n x d momentum buffers
+    z: np.ndarray                      # n x d de-biased parameters
+    transit_x: deque = field(default_factory=deque)   # tau in-flight (n x d) messages, oldest first
+    transit_w: deque = field(default_factory=deque)   # tau in-flight (n) weight messages
+
+
+def init_state(x0, tau: int = 0) -> SGPState:
+    """Alg. 1 'Require' line: w = 1, z = x; Alg. 3: u = 0; virtual nodes hold 0."""
+    x = np.array(x0, dtype=np.float64)
+    n, d = x.shape
+    st = SGPState(x=x, w=np.ones(n), u=np.zeros((n, d)), z=x.copy())
+    for _ in range(tau):
+        st.transit_x.append(np.zeros((n, d)))
+        st.transit_w.append(np.zeros(n))
+    return st
+
+
+def local_update(x, u, g, lr, momentum=0.0, nesterov=True, weight_decay=0.0):
+    """Half step x^(k+1/2) on the numerators (Alg. 1 line 4 / Alg. 3 lines 4-5).
+
+    Returns (h, u_next) with h = x^(k+1/2).
+    """
+    g = np.asarray(g, dtype=np.float64)
+    if weight_decay != 0.0:
+        g = g + weight_decay * x
+    if momentum != 0.0:
+        u_next = momentum * u + g                      # Alg. 3 line 4
+        if nesterov:
+            s = momentum * u_next + g                  # Alg. 3 line 5
+        else:
+            s = u_next                                 # classical (heavy-ball) momentum
+    else:
+        u_next = u
+        s = g                                          # Alg. 1 line 4
+    h = x - lr * s
+    return h, u_next
+
+
+def mix(P, h, w):
+    """One PushSum iteration, no delay (Alg. 1 lines 6-7): x' = P h, w' = P w."""
+    return P @ h, P @ w
+
+
+def mix_delayed(P, h, w, transit_x, transit_w):
+    """One PushSum iteration where every off-diagonal message is tau steps late.
+
+    Block form of the augmented matrix: P~_0 = diag(P) acts now, P~_tau =
+    P - diag(P) enters the far end of the delay chain, virtual nodes forward.
+    ``transit_*`` hold exactly tau messages, oldest first.
+    """
+    diag = np.diag(P)
+    off = P - np.diag(diag)
+    arriving_x = transit_x.popleft()
+    arriving_w = transit_w.popleft()
+    x_next = diag[:, None] * h + arriving_x            # Alg. 2 lines 7, 21
+    w_next = diag * w + arriving_w                     # Alg. 2 lines 8, 22 (accumulating)
+    transit_x.append(off @ h)                          # Alg. 2 line 6 (non-blocking send)
+    transit_w.append(off @ w)
+    return x_next, w_next
+
+
+def sgp_step(st: SGPState, g, P, lr, momentum=0.0, nesterov=True, weight_decay=0.0) -> SGPState:
+    """One full SGP iteration in place on ``st`` (gradient g was taken at st.z)."""
+    h, st.u = local_update(st.x, st.u, g, lr, momentum, nesterov, weight_decay)
+    if len(st.transit_x) == 0:
+        st.x, st.w = mix(P, h, st.w)
+    else:
+        st.x, st.w = mix_delayed(P, h, st.w, st.transit_x, st.transit_w)
+    st.z = st.x / st.w[:, None]                        # Alg. 1 line 8
+    return st
+
+
+def sgp_run(x0, K, P_of_k, grad_of_k, lr, momentum=0.0, nesterov=True, weight_decay=0.0,
+            tau=0, history=None) -> SGPState:
+    """K iterations k = 0 .. K-1.
+
+    ``P_of_k(k)`` returns the dense mixing matrix of step k; ``grad_of_k(k, z)``
+    returns the n x d stochastic gradients evaluated at the de-biased ``z``.
+    If ``history`` is a list, a snapshot (x, w, u, z) is appended after every step.
+    """
+    st = init_state(x0, tau)
+    for k in range(K):
+        g = grad_of_k(k, st.z)
+        sgp_step(st, g, P_of_k(k), lr, momentum, nesterov, weight_decay)
+        if history is not None:
+            history.append((st.x.copy(), st.w.copy(), st.u.copy(), st.z.copy()))
+    return st
+
+
+def debias(x, w):
+    """z_i = x_i / w_i (Alg. 1 line 8)."""
+    return np.asarray(x, dtype=np.float64) / np.asarray(w, dtype=np.float64)[:, None]
+
+
+def total_mass(st: SGPState):
+    """(sum of x over real and in-transit nodes, same for w): conserved by the mix."""
+    sx = st.x.sum(axis=0)
+    sw = st.w.sum()
+    for mx, mw in zip(st.transit_x, st.transit_w):
+        sx = sx + mx.sum(axis=0)
+        sw = sw + mw.sum()
+    return sx, sw
