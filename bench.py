@@ -1,0 +1,324 @@
+#!/usr/bin/env python
+"""Benchmark of the fused SGP step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload resnet50] [--impl ours|reference]
+
+One "step" is one whole SGP iteration (local Nesterov update, PushSum mix, weight mix, de-bias) for
+all n simulated nodes.  The default workload is the ResNet-50-sized run: n = 32 nodes, d = 25,557,032
+parameters, one-peer exponential graph, Nesterov 0.9, weight decay 1e-4, Z written (24 algorithmic
+bytes per node-parameter).  Prints ONE JSON line on rank 0.
+
+With N > 1 every rank runs an independent replica of the same workload on its own GPU (the path has
+no exchange step between GPUs); `value` is the sum over ranks divided by the slowest rank's time.
+`--impl reference` times the float64 CPU oracle on a bounded column sample instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "node_param_updates_per_sec"
+UNIT = "updates/s"
+FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused step kernel, from the ncu capture
+# summarised under profiles/ (captured on a column-scaled case and scaled by the units processed).
+NCU_TRAFFIC_BYTES = {}
+
+
+def bytes_per_update(w, write_z=True) -> int:
+    """Algorithmic HBM bytes per node-parameter per step (fp32, in place)."""
+    b = 4 * (2 + 1)                       # read x, g; write x
+    if w.momentum != 0.0:
+        b += 8                            # read u, write u
+    if write_z:
+        b += 4
+    if w.tau > 0:
+        b += 8                            # read + write one ring slot
+    return b
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Polls NVML for SM clock and throttle reasons while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self._armed = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self._nv = None
+
+    def _run(self):
+        nv = self._nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+        }
+        while not self._stop.is_set():
+            try:
+                mhz = nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self._h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h)
+                if self._armed:
+                    self.samples.append(mhz)
+                    for k, bit in names.items():
+                        if mask & bit:
+                            self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def start(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def arm(self, on: bool):
+        self._armed = on
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join(timeout=1.0)
+
+    def summary(self):
+        s = sorted(self.samples)
+        return {"sm_mhz": (s[len(s) // 2] if s else None), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(s)}
+
+
+def oracle_sample_run(w, sample_cols: int, steps: int, warmup: int):
+    """Times the float64 oracle, as it stands, on the first `sample_cols` columns of the workload.
+    Returns (seconds per step, BLAS threads)."""
+    import numpy as np
+    import torch
+    from oracle import sgp as osgp
+    from paper_1811_10792_b200 import inputs
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    from parity_util import oracle_P_of_k
+
+    x0 = inputs.initial_x(w, device="cpu", d=sample_cols).numpy().astype(np.float64)
+    G = torch.empty((w.n, sample_cols), dtype=torch.float32)
+    grads = [inputs.gradient(w, k, G).numpy().astype(np.float64) for k in range(min(4, steps + warmup))]
+    P_of_k = oracle_P_of_k(w)
+    st = osgp.init_state(x0, w.tau)
+    for k in range(warmup):
+        osgp.sgp_step(st, grads[k % len(grads)], P_of_k(k), w.lr, w.momentum, w.nesterov, w.weight_decay)
+    t0 = time.perf_counter()
+    for k in range(warmup, warmup + steps):
+        osgp.sgp_step(st, grads[k % len(grads)], P_of_k(k), w.lr, w.momentum, w.nesterov, w.weight_decay)
+    dt = (time.perf_counter() - t0) / steps
+    threads = 1
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        pass
+    return dt, threads
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    sample_cols = min(w.d, 1 << 18)
+    dt, threads = oracle_sample_run(w, sample_cols, args.steps, args.warmup)
+    value = w.n * sample_cols / dt
+    sample = f"float64 numpy oracle, columns [0, {sample_cols}) of {w.d} ({100.0 * sample_cols / w.d:.2f}%), all {w.n} nodes"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": workload_config(w, extra={"sample_cols": sample_cols}),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(w, extra=None):
+    cfg = {"workload": f"{w.name}: n={w.n} nodes x d={w.d} fp32 parameters, {w.peers}-peer exponential digraph"
+                       if w.graph == "exp" else f"{w.name}: n={w.n} x d={w.d}, {w.graph} digraph",
+           "n": w.n, "d": w.d, "graph": w.graph, "peers": w.peers, "tau": w.tau, "lr": w.lr, "momentum": w.momentum,
+           "nesterov": w.nesterov, "weight_decay": w.weight_decay, "writes_z": True,
+           "l2_policy": "inputs larger than L2 (every array >= 3 GB, streamed once per step)"}
+    if extra:
+        cfg.update(extra)
+    return cfg
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="resnet50")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--d", type=int, default=0, help="override the parameter count (profiling on a small case)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--option", action="append", default=[], help="key=value passed to sgp_set_option")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    from paper_1811_10792_b200 import inputs
+    w = inputs.WORKLOADS[args.workload]
+    if args.d > 0:
+        w = w.scaled(args.d)
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_1811_10792_b200 import binding     # raises if the CUDA library is missing: no fallback
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    from parity_util import graph_desc
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (there is no CPU path)")
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    n, d, K, Wm = w.n, w.d, args.steps, args.warmup
+    free_b, _total_b = torch.cuda.mem_get_info()
+    arr_bytes = 4 * n * d
+    n_state = 3 + (1 if w.tau else 0)                       # X, M, Z (+ ring inside the handle)
+    pool = max(1, min(K, int((free_b * 0.6 - n_state * arr_bytes) // arr_bytes)))
+    X = inputs.initial_x(w, device=dev).contiguous()
+    M = torch.zeros_like(X) if w.momentum != 0.0 else None
+    Z = torch.empty_like(X)
+    Wt = torch.ones(n, device=dev)
+    Gs = []
+    for k in range(pool):
+        G = torch.empty_like(X)
+        inputs.gradient(w, k, G)
+        Gs.append(G)
+    h = binding.Sgp(n, d, graph_desc(w, binding), tau=w.tau)
+    for kv in args.option:
+        key, val = kv.split("=")
+        h.set_option(key, int(val))
+
+    def step(k):
+        h.step(X, Wt, M, Gs[k % pool], Z, k, w.lr, w.momentum, w.weight_decay, w.nesterov)
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    for k in range(Wm):
+        step(k)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(K + 1)]
+    sampler.arm(True)
+    for i in range(K):
+        evs[i].record()
+        step(Wm + i)
+    evs[K].record()
+    torch.cuda.synchronize()
+    sampler.arm(False)
+    if world > 1:
+        dist.barrier()
+    total_ms = evs[0].elapsed_time(evs[K])
+    per_step_ms = [evs[i].elapsed_time(evs[i + 1]) for i in range(K)]
+    assert h.device_status() == 0
+    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    max_ms = float(t.item())
+    value = world * n * d * K / (max_ms * 1e-3)
+
+    # ---- end to end through the host-buffer entry point (gradients in, de-biased parameters out)
+    e2e = None
+    if not args.no_e2e:
+        hG = torch.empty((n, d), dtype=torch.float32, pin_memory=True)
+        hZ = torch.empty((n, d), dtype=torch.float32, pin_memory=True)
+        hG.copy_(Gs[0])
+        dG = Gs[0]
+        torch.cuda.synchronize()
+        e2e_steps = K
+        h.step_host(X, Wt, M, hG, hZ, dG, Z, Wm + K, w.lr, w.momentum, w.weight_decay, w.nesterov)   # warm
+        if world > 1:
+            dist.barrier()
+        t0 = time.perf_counter()
+        for i in range(e2e_steps):
+            h.step_host(X, Wt, M, hG, hZ, dG, Z, Wm + K + 1 + i, w.lr, w.momentum, w.weight_decay, w.nesterov)
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        t2 = torch.tensor([dt], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(t2, op=dist.ReduceOp.MAX)
+        e2e = {"value": world * n * d * e2e_steps / float(t2.item()), "unit": UNIT,
+               "h2d_bytes_per_step": arr_bytes, "d2h_bytes_per_step": arr_bytes, "steps": e2e_steps,
+               "ms_per_step": float(t2.item()) * 1e3 / e2e_steps}
+        del hG, hZ
+    sampler.stop()
+
+    if rank == 0:
+        peak, peak_kind = measured_peak()
+        bpu = bytes_per_update(w)
+        kern_ms = sum(per_step_ms) / len(per_step_ms)
+        achieved = bpu * n * d / (kern_ms * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                    "traffic": NCU_TRAFFIC_BYTES.get(w.name), "peak_kind": f"of {peak_kind}",
+                    "kernel": "sgp_step (fused update + mix + de-bias)", "algorithmic_bytes_per_launch": bpu * n * d,
+                    "kernel_ms": kern_ms, "frac_of_nominal_8TBps": achieved / NOMINAL_HBM_GBS}
+        cpu = None
+        if not args.no_cpu_baseline:
+            sample_cols = min(d, 1 << 20)
+            dt, threads = oracle_sample_run(w, sample_cols, steps=8, warmup=1)
+            cpu = {"value": n * sample_cols / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
+                   "sample": f"8 steps of the float64 numpy oracle on columns [0, {sample_cols}) "
+                             f"({100.0 * sample_cols / d:.2f}% of d), all {n} nodes; host has "
+                             f"{len(os.sched_getaffinity(0))} usable cores"}
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+            "ms_per_step": max_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": workload_config(w, extra={"gradient_pool": pool, "parallelism": f"replicas x{world}"}),
+            "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": K, "clocks": sampler.summary(),
+        }
+        print(json.dumps(line), flush=True)
+    h.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

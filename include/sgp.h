@@ -1,0 +1,184 @@
+/*
+ * sgp.h -- C ABI of the fused Stochastic Gradient Push (SGP) step for n simulated nodes
+ *          stacked on one NVIDIA B200 (sm_100a).
+ *
+ * State (all fp32, owned by the caller, DEVICE memory unless a name starts with h_):
+ *   X  n x ld   push-sum numerators x_i            (row i = node i, ld >= d floats between rows)
+ *   W  n        push-sum weights w_i               (w_i^(0) = 1)
+ *   M  n x ld   momentum buffers u_i               (never mixed; u^(0) = 0)
+ *   G  n x ld   stochastic gradients of step k, evaluated by the caller at Z
+ *   Z  n x ld   de-biased parameters z_i = x_i / w_i
+ * Convention for the mixing matrix P^(k): p_ij is the weight RECEIVER i applies to SENDER j
+ * (rows = receivers, columns = senders), every node is its own in/out-neighbour, columns sum to 1
+ * (Sec. 2 "Approximate distributed averaging"; supplementary "Modeling message delays").
+ *
+ * Every function returns an int status (SGP_OK = 0, negative = error), never throws, aborts or prints.
+ * Kernels are enqueued on the caller's stream (a cudaStream_t passed as void*) and the calls return
+ * without synchronising unless stated.  No call falls back to the CPU.
+ */
+#ifndef SGP_H_
+#define SGP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SGP_OK            0
+#define SGP_ERR_ARG      -1   /* bad size, null pointer, misaligned pointer, k < 0, ...               */
+#define SGP_ERR_GRAPH    -2   /* schedule is not a valid column-stochastic digraph with self-loops    */
+#define SGP_ERR_CUDA     -3   /* a CUDA runtime call failed; see sgp_last_cuda_error                  */
+#define SGP_ERR_ALLOC    -4   /* host or device allocation failed                                     */
+#define SGP_ERR_STATE    -5   /* call not valid for this handle (e.g. ring export with tau = 0)       */
+#define SGP_ERR_DEVICE   -6   /* a kernel reported a bounded wait that ran out (status word non-zero) */
+
+#define SGP_MAX_NODES 256     /* n <= 256: one CTA keeps all n rows of a column tile on chip          */
+
+/* Which time-varying digraph the schedule compiler expands. */
+typedef enum sgp_graph_kind {
+  SGP_GRAPH_EXP_PEERS     = 0, /* App. A directed exponential graph, `peers` out-neighbours per step */
+  SGP_GRAPH_COMPLETE      = 1, /* every entry 1/n (Sec. 3: equivalent to AllReduce parallel SGD)     */
+  SGP_GRAPH_RANDOM_OUTDEG = 2, /* hashed random digraph, out-degree ~ U{1..min(max_outdeg, n-1)}     */
+  SGP_GRAPH_CUSTOM        = 3  /* explicit edge list with per-edge weights                           */
+} sgp_graph_kind;
+
+/*
+ * Schedule descriptor (plain data, HOST memory, read only during the call that takes it).
+ *  EXP_PEERS : at step k node i sends to (i + 2^((k+t) mod L)) mod n, t = 0..peers-1, with
+ *              L = floor(log2(n-1)) + 1 hop distances (App. A); weights 1/|N_out| incl. self (App. C).
+ *  RANDOM    : `num_steps` distinct steps, then the schedule repeats; draws are a keyed integer
+ *              hash of (seed, step, node, draw) so that independent implementations agree bit for bit.
+ *  CUSTOM    : num_edges quadruples (edge_step, edge_sender, edge_receiver, edge_weight); self-loops are
+ *              listed explicitly; steps 0..num_steps-1, repeating.  Rejected with SGP_ERR_GRAPH if an
+ *              index is out of range, an edge is duplicated, a weight is not finite and > 0, a
+ *              self-loop is missing, or a column does not sum to 1 within 4*deg*2^-24.
+ */
+typedef struct sgp_graph_desc {
+  int32_t  kind;         /* sgp_graph_kind                                         */
+  int32_t  peers;        /* EXP_PEERS: >= 1 (paper uses 1 and 2)                   */
+  int32_t  max_outdeg;   /* RANDOM_OUTDEG: >= 1                                    */
+  int32_t  reserved;     /* must be 0                                              */
+  uint64_t seed;         /* RANDOM_OUTDEG                                          */
+  int64_t  num_steps;    /* RANDOM_OUTDEG, CUSTOM: period of the schedule (>= 1)   */
+  const int32_t *edge_step;      /* CUSTOM only, host arrays of num_edges entries  */
+  const int32_t *edge_sender;
+  const int32_t *edge_receiver;
+  const float   *edge_weight;
+  int64_t  num_edges;
+} sgp_graph_desc;
+
+/* ---------------------------------------------------------------------------------------------
+ * Graph-schedule compiler (host only; needs no GPU).  Turns the time-varying digraph into, for
+ * every step of one period, the in-neighbour lists of P^(k) in CSR form: row i lists the senders j
+ * with p_ij != 0 in ascending j (self in its sorted place) and the fp32 weights p_ij.  For the
+ * uniform kinds p_ij = (float)(1.0 / |N_out_j|) (App. C).  Defines the mix x_i' = sum_j p_ij x_j
+ * of Alg. 1 line 6.  The returned object is owned by the caller until sgp_schedule_destroy.
+ * ------------------------------------------------------------------------------------------- */
+typedef struct sgp_schedule sgp_schedule;
+
+int sgp_schedule_compile(sgp_schedule **out, int n, const sgp_graph_desc *g);
+int sgp_schedule_destroy(sgp_schedule *s);
+/* Number of distinct steps; step k uses slot k mod period. */
+int sgp_schedule_period(const sgp_schedule *s, int64_t *period);
+/* Non-zeros of P^(k). */
+int sgp_schedule_nnz(const sgp_schedule *s, int64_t k, int64_t *nnz);
+/* Copies step k's CSR into HOST arrays rowptr[n+1], col[cap], val[cap]; SGP_ERR_ARG if cap < nnz. */
+int sgp_schedule_get(const sgp_schedule *s, int64_t k, int32_t *rowptr, int32_t *col, float *val,
+                     int64_t cap, int64_t *nnz);
+
+/* ---------------------------------------------------------------------------------------------
+ * Handle: compiled schedule uploaded to the device, the ring of delayed messages (tau > 0) and a
+ * few words of launch scratch.  Problem statement: Eq. 1 (n nodes, parameters in R^d).
+ * ------------------------------------------------------------------------------------------- */
+typedef struct sgp_handle sgp_handle;
+
+#define SGP_FLAG_NONE 0u
+
+/*
+ * sgp_create: n nodes (1..SGP_MAX_NODES), d parameters per node, ld >= d the row pitch in floats of
+ * every n x ld array later passed to this handle, graph schedule g (compiled here), tau >= 0 the
+ * fixed message delay of Overlap SGP (Alg. 2; tau = 0 is Alg. 1).  For tau > 0 the handle allocates
+ * and zeroes a ring of tau slots of n x ld floats plus tau x n weights (virtual nodes start at
+ * zero).  Uses the current CUDA device.  Synchronises.  On error *out is NULL.
+ */
+int sgp_create(sgp_handle **out, int n, int64_t d, int64_t ld, const sgp_graph_desc *g, int tau,
+               unsigned flags);
+/* Frees everything the handle owns.  Synchronises the device.  NULL is accepted. */
+int sgp_destroy(sgp_handle *h);
+/* The handle's compiled schedule (owned by the handle; valid until sgp_destroy). */
+int sgp_get_schedule(const sgp_handle *h, const sgp_schedule **s);
+
+/*
+ * sgp_step: one whole SGP iteration k for all n nodes, in ONE pass over HBM (Alg. 1 lines 4-8 with
+ * the update of Alg. 3 lines 4-5; Alg. 2 for tau > 0):
+ *     g~  = G + weight_decay * X
+ *     momentum != 0:  M <- momentum*M + g~ ;  s = momentum*M + g~ (nesterov) or M (otherwise)
+ *     momentum == 0:  s = g~                          (d_M may be NULL and is not touched)
+ *     h   = X - lr * s
+ *     tau == 0:  X_i <- sum_j p_ij h_j ,  W_i <- sum_j p_ij W_j           (CSR order, fp32 FMA)
+ *     tau  > 0:  X_i <- p_ii h_i + ring[k mod tau]_i ; ring[k mod tau]_i <- sum_{j != i} p_ij h_j
+ *                (same for W): a message sent at step k is consumed by step k + tau
+ *     Z_i <- X_i * (1 / W_i)          if d_Z != NULL  (reciprocal rounded once per node)
+ * X, W, M are updated in place; G is only read; Z is only written.  All arrays n x ld fp32 device
+ * memory except W (n floats).  Arrays must not overlap.  If every pointer is 16-byte aligned and
+ * ld is a multiple of 4 the 128-bit path runs, otherwise a scalar path (slower, same results).
+ * k >= 0 selects the schedule slot k mod period and the ring slot k mod tau; for tau > 0 the caller
+ * must present k = 0, 1, 2, ... in order.  Asynchronous on `stream`; calls on the same handle must
+ * be stream-ordered with respect to each other.
+ */
+int sgp_step(sgp_handle *h, float *d_X, float *d_W, float *d_M, const float *d_G, float *d_Z,
+             int64_t k, float lr, float momentum, float weight_decay, int nesterov, void *stream);
+
+/* sgp_debias: Z_i = X_i * (1 / W_i) for all nodes (Alg. 1 line 8), one pass.  X may equal Z. */
+int sgp_debias(sgp_handle *h, const float *d_X, const float *d_W, float *d_Z, void *stream);
+
+/*
+ * sgp_step_host: the same iteration for callers whose gradients and parameters live in HOST memory.
+ * h_G (read) and h_Z (written, may be NULL) are n x ld host arrays, ideally page-locked; X, W, M stay
+ * resident on the device; d_G and d_Z are device staging arrays of n x ld floats supplied by the
+ * caller.  The columns are cut into chunks; chunk c's host->device copy, its fused step and its
+ * device->host copy overlap with the neighbouring chunks on the handle's two internal streams.
+ * Returns after everything has completed (synchronises).  chunk_cols <= 0 picks a default.
+ */
+int sgp_step_host(sgp_handle *h, float *d_X, float *d_W, float *d_M, const float *h_G, float *h_Z,
+                  float *d_G, float *d_Z, int64_t k, float lr, float momentum, float weight_decay,
+                  int nesterov, int64_t chunk_cols);
+
+/* Zeroes the delay ring (messages in transit are dropped: use only to restart a run). */
+int sgp_reset(sgp_handle *h, void *stream);
+/* Checkpointing of the in-transit messages: d_ring_x is tau*n*ld floats, d_ring_w is tau*n floats
+ * (device memory), slot-major.  SGP_ERR_STATE if tau == 0. */
+int sgp_ring_export(sgp_handle *h, float *d_ring_x, float *d_ring_w, void *stream);
+int sgp_ring_import(sgp_handle *h, const float *d_ring_x, const float *d_ring_w, void *stream);
+
+/*
+ * sgp_check: invariants of column-stochastic mixing (Sec. 2; delay model: mass in transit counts).
+ * Writes to HOST h_stats[4]: { sum_i W_i + sum of ring weights (should equal n), min_i W_i,
+ * number of non-finite entries of X, sum over all entries of X and the ring }.  Synchronises.
+ */
+int sgp_check(sgp_handle *h, const float *d_X, const float *d_W, double *h_stats, void *stream);
+
+/*
+ * Tuning knobs for experiments (defaults are chosen per problem shape):
+ *   "variant"      0 = automatic, 1 = register-staged kernel, 2 = bulk-copy (TMA) pipelined kernel
+ *   "tile_cols"    columns per tile (multiple of 4; 0 = automatic)
+ *   "ctas_per_sm"  persistent CTAs per SM (0 = automatic)
+ * Unknown keys or unsupported values return SGP_ERR_ARG and change nothing.
+ */
+int sgp_set_option(sgp_handle *h, const char *key, int64_t value);
+int sgp_get_option(const sgp_handle *h, const char *key, int64_t *value);
+
+/* Reads the handle's device status word (0 = no kernel ever gave up a bounded wait).  Synchronises. */
+int sgp_device_status(sgp_handle *h, unsigned *status);
+/* cudaError_t value latched by the last call that returned SGP_ERR_CUDA on this handle (0 if none). */
+int sgp_last_cuda_error(const sgp_handle *h);
+const char *sgp_strerror(int code);
+/* Library version as major*10000 + minor*100 + patch. */
+int sgp_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SGP_H_ */

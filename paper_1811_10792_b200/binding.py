@@ -1,0 +1,286 @@
+"""ctypes binding of libsgp.so: argument marshalling only, same names as include/sgp.h.
+
+Every step of the SGP iteration runs inside the CUDA library; nothing here computes.  The library
+is loaded from this package's directory and the import fails loudly if it is missing: there is no
+CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_PKG_DIR = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG_DIR, "libsgp.so")
+
+SGP_OK, SGP_ERR_ARG, SGP_ERR_GRAPH, SGP_ERR_CUDA, SGP_ERR_ALLOC, SGP_ERR_STATE, SGP_ERR_DEVICE = 0, -1, -2, -3, -4, -5, -6
+SGP_MAX_NODES = 256
+SGP_GRAPH_EXP_PEERS, SGP_GRAPH_COMPLETE, SGP_GRAPH_RANDOM_OUTDEG, SGP_GRAPH_CUSTOM = 0, 1, 2, 3
+
+# every symbol include/sgp.h declares
+EXPORTS = [
+    "sgp_schedule_compile", "sgp_schedule_destroy", "sgp_schedule_period", "sgp_schedule_nnz", "sgp_schedule_get",
+    "sgp_create", "sgp_destroy", "sgp_get_schedule", "sgp_step", "sgp_debias", "sgp_step_host", "sgp_reset",
+    "sgp_ring_export", "sgp_ring_import", "sgp_check", "sgp_set_option", "sgp_get_option", "sgp_device_status",
+    "sgp_last_cuda_error", "sgp_strerror", "sgp_version",
+]
+
+
+class SgpError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        self.code = code
+        super().__init__(f"{what}: {strerror(code)} ({code})")
+
+
+class sgp_graph_desc(C.Structure):
+    _fields_ = [
+        ("kind", C.c_int32), ("peers", C.c_int32), ("max_outdeg", C.c_int32), ("reserved", C.c_int32),
+        ("seed", C.c_uint64), ("num_steps", C.c_int64),
+        ("edge_step", C.POINTER(C.c_int32)), ("edge_sender", C.POINTER(C.c_int32)),
+        ("edge_receiver", C.POINTER(C.c_int32)), ("edge_weight", C.POINTER(C.c_float)),
+        ("num_edges", C.c_int64),
+    ]
+
+
+def _load() -> C.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_1811_10792_b200.build` "
+            "(there is no fallback implementation)")
+    lib = C.CDLL(LIB_PATH)
+    vp, i64, f32, i32 = C.c_void_p, C.c_int64, C.c_float, C.c_int
+    sig = {
+        "sgp_schedule_compile": [C.POINTER(vp), i32, C.POINTER(sgp_graph_desc)],
+        "sgp_schedule_destroy": [vp],
+        "sgp_schedule_period": [vp, C.POINTER(i64)],
+        "sgp_schedule_nnz": [vp, i64, C.POINTER(i64)],
+        "sgp_schedule_get": [vp, i64, vp, vp, vp, i64, C.POINTER(i64)],
+        "sgp_create": [C.POINTER(vp), i32, i64, i64, C.POINTER(sgp_graph_desc), i32, C.c_uint],
+        "sgp_destroy": [vp],
+        "sgp_get_schedule": [vp, C.POINTER(vp)],
+        "sgp_step": [vp, vp, vp, vp, vp, vp, i64, f32, f32, f32, i32, vp],
+        "sgp_debias": [vp, vp, vp, vp, vp],
+        "sgp_step_host": [vp, vp, vp, vp, vp, vp, vp, vp, i64, f32, f32, f32, i32, i64],
+        "sgp_reset": [vp, vp],
+        "sgp_ring_export": [vp, vp, vp, vp],
+        "sgp_ring_import": [vp, vp, vp, vp],
+        "sgp_check": [vp, vp, vp, C.POINTER(C.c_double), vp],
+        "sgp_set_option": [vp, C.c_char_p, i64],
+        "sgp_get_option": [vp, C.c_char_p, C.POINTER(i64)],
+        "sgp_device_status": [vp, C.POINTER(C.c_uint)],
+        "sgp_last_cuda_error": [vp],
+        "sgp_version": [],
+    }
+    for name, args in sig.items():
+        fn = getattr(lib, name)
+        fn.argtypes = args
+        fn.restype = C.c_int
+    lib.sgp_strerror.argtypes = [C.c_int]
+    lib.sgp_strerror.restype = C.c_char_p
+    return lib
+
+
+_lib = _load()
+
+
+def lib() -> C.CDLL:
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return _lib.sgp_strerror(code).decode()
+
+
+def _check(code: int, what: str) -> None:
+    if code != SGP_OK:
+        raise SgpError(code, what)
+
+
+class GraphDesc:
+    """Owns the host arrays behind a sgp_graph_desc."""
+
+    def __init__(self, kind: int, peers: int = 1, max_outdeg: int = 4, seed: int = 0, num_steps: int = 0,
+                 edges=None):
+        self.c = sgp_graph_desc()
+        self.c.kind, self.c.peers, self.c.max_outdeg = kind, peers, max_outdeg
+        self.c.reserved, self.c.seed, self.c.num_steps = 0, seed, num_steps
+        self._keep = []
+        if edges is not None:
+            step, sender, receiver, weight = edges
+            arrs = [np.ascontiguousarray(step, dtype=np.int32), np.ascontiguousarray(sender, dtype=np.int32),
+                    np.ascontiguousarray(receiver, dtype=np.int32), np.ascontiguousarray(weight, dtype=np.float32)]
+            self._keep = arrs
+            self.c.edge_step = arrs[0].ctypes.data_as(C.POINTER(C.c_int32))
+            self.c.edge_sender = arrs[1].ctypes.data_as(C.POINTER(C.c_int32))
+            self.c.edge_receiver = arrs[2].ctypes.data_as(C.POINTER(C.c_int32))
+            self.c.edge_weight = arrs[3].ctypes.data_as(C.POINTER(C.c_float))
+            self.c.num_edges = len(arrs[0])
+
+    @staticmethod
+    def exp_peers(peers: int = 1) -> "GraphDesc":
+        return GraphDesc(SGP_GRAPH_EXP_PEERS, peers=peers)
+
+    @staticmethod
+    def complete() -> "GraphDesc":
+        return GraphDesc(SGP_GRAPH_COMPLETE)
+
+    @staticmethod
+    def random_outdeg(seed: int, num_steps: int, max_outdeg: int = 4) -> "GraphDesc":
+        return GraphDesc(SGP_GRAPH_RANDOM_OUTDEG, max_outdeg=max_outdeg, seed=seed, num_steps=num_steps)
+
+    @staticmethod
+    def custom(num_steps: int, step, sender, receiver, weight) -> "GraphDesc":
+        return GraphDesc(SGP_GRAPH_CUSTOM, num_steps=num_steps, edges=(step, sender, receiver, weight))
+
+
+class _ScheduleView:
+    """Read access to a compiled schedule (host arrays)."""
+
+    def __init__(self, ptr, n):
+        self._ptr, self.n = ptr, n
+
+    @property
+    def period(self) -> int:
+        v = C.c_int64()
+        _check(_lib.sgp_schedule_period(self._ptr, C.byref(v)), "sgp_schedule_period")
+        return v.value
+
+    def nnz(self, k: int) -> int:
+        v = C.c_int64()
+        _check(_lib.sgp_schedule_nnz(self._ptr, k, C.byref(v)), "sgp_schedule_nnz")
+        return v.value
+
+    def get(self, k: int):
+        """(rowptr int32[n+1], col int32[nnz], val float32[nnz]) of step k."""
+        nnz = self.nnz(k)
+        rowptr = np.empty(self.n + 1, dtype=np.int32)
+        col = np.empty(max(nnz, 1), dtype=np.int32)
+        val = np.empty(max(nnz, 1), dtype=np.float32)
+        out = C.c_int64()
+        _check(_lib.sgp_schedule_get(self._ptr, k, rowptr.ctypes.data, col.ctypes.data, val.ctypes.data, nnz,
+                                     C.byref(out)), "sgp_schedule_get")
+        return rowptr, col[:nnz], val[:nnz]
+
+
+class Schedule(_ScheduleView):
+    """sgp_schedule_compile: host-only graph-schedule compiler (needs no GPU)."""
+
+    def __init__(self, n: int, graph: GraphDesc):
+        ptr = C.c_void_p()
+        _check(_lib.sgp_schedule_compile(C.byref(ptr), n, C.byref(graph.c)), "sgp_schedule_compile")
+        super().__init__(ptr, n)
+
+    def close(self):
+        if getattr(self, "_ptr", None):
+            _lib.sgp_schedule_destroy(self._ptr)
+            self._ptr = None
+
+    def __del__(self):
+        self.close()
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream_ptr(stream):
+    import torch
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+class Sgp:
+    """sgp_create / sgp_step / sgp_debias ... on torch CUDA tensors (fp32, row pitch ld)."""
+
+    def __init__(self, n: int, d: int, graph: GraphDesc, tau: int = 0, ld: int | None = None, flags: int = 0):
+        self.n, self.d, self.ld, self.tau = n, d, (d if ld is None else ld), tau
+        self._h = C.c_void_p()
+        _check(_lib.sgp_create(C.byref(self._h), n, d, self.ld, C.byref(graph.c), tau, flags), "sgp_create")
+
+    def close(self):
+        if getattr(self, "_h", None):
+            _lib.sgp_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        self.close()
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    @property
+    def schedule(self) -> _ScheduleView:
+        p = C.c_void_p()
+        _check(_lib.sgp_get_schedule(self._h, C.byref(p)), "sgp_get_schedule")
+        return _ScheduleView(p, self.n)
+
+    def _check_mat(self, t, name, allow_none=False):
+        import torch
+        if t is None:
+            if allow_none:
+                return
+            raise ValueError(f"{name} is required")
+        if t.dtype != torch.float32 or not t.is_cuda:
+            raise ValueError(f"{name} must be a float32 CUDA tensor")
+        if t.dim() != 2 or t.shape[0] != self.n or t.shape[1] != self.d or t.stride(1) != 1 or \
+                (self.n > 1 and t.stride(0) != self.ld):
+            raise ValueError(f"{name} must be n x d with row pitch ld={self.ld}")
+
+    def step(self, X, W, M, G, Z, k: int, lr: float, momentum: float = 0.0, weight_decay: float = 0.0,
+             nesterov: bool = True, stream=None) -> None:
+        self._check_mat(X, "X")
+        self._check_mat(G, "G")
+        self._check_mat(M, "M", allow_none=(momentum == 0.0))
+        self._check_mat(Z, "Z", allow_none=True)
+        _check(_lib.sgp_step(self._h, _ptr(X), _ptr(W), _ptr(M), _ptr(G), _ptr(Z), k, lr, momentum, weight_decay,
+                             int(bool(nesterov)), _stream_ptr(stream)), "sgp_step")
+
+    def debias(self, X, W, Z, stream=None) -> None:
+        self._check_mat(X, "X")
+        self._check_mat(Z, "Z")
+        _check(_lib.sgp_debias(self._h, _ptr(X), _ptr(W), _ptr(Z), _stream_ptr(stream)), "sgp_debias")
+
+    def step_host(self, X, W, M, h_G, h_Z, d_G, d_Z, k: int, lr: float, momentum: float = 0.0,
+                  weight_decay: float = 0.0, nesterov: bool = True, chunk_cols: int = 0) -> None:
+        """h_G / h_Z are host (ideally pinned) tensors; everything else lives on the device."""
+        _check(_lib.sgp_step_host(self._h, _ptr(X), _ptr(W), _ptr(M), _ptr(h_G), _ptr(h_Z), _ptr(d_G), _ptr(d_Z),
+                                  k, lr, momentum, weight_decay, int(bool(nesterov)), chunk_cols), "sgp_step_host")
+
+    def reset(self, stream=None) -> None:
+        _check(_lib.sgp_reset(self._h, _stream_ptr(stream)), "sgp_reset")
+
+    def ring_export(self, ring_x, ring_w, stream=None) -> None:
+        _check(_lib.sgp_ring_export(self._h, _ptr(ring_x), _ptr(ring_w), _stream_ptr(stream)), "sgp_ring_export")
+
+    def ring_import(self, ring_x, ring_w, stream=None) -> None:
+        _check(_lib.sgp_ring_import(self._h, _ptr(ring_x), _ptr(ring_w), _stream_ptr(stream)), "sgp_ring_import")
+
+    def check(self, X, W, stream=None):
+        """(sum of weights incl. in transit, min weight, non-finite count in X, sum of X incl. in transit)."""
+        out = (C.c_double * 4)()
+        _check(_lib.sgp_check(self._h, _ptr(X), _ptr(W), out, _stream_ptr(stream)), "sgp_check")
+        return tuple(out)
+
+    def set_option(self, key: str, value: int) -> None:
+        _check(_lib.sgp_set_option(self._h, key.encode(), value), "sgp_set_option")
+
+    def get_option(self, key: str) -> int:
+        v = C.c_int64()
+        _check(_lib.sgp_get_option(self._h, key.encode(), C.byref(v)), "sgp_get_option")
+        return v.value
+
+    def device_status(self) -> int:
+        v = C.c_uint()
+        _check(_lib.sgp_device_status(self._h, C.byref(v)), "sgp_device_status")
+        return v.value
+
+    def last_cuda_error(self) -> int:
+        return _lib.sgp_last_cuda_error(self._h)
+
+
+def version() -> int:
+    return _lib.sgp_version()

@@ -1,0 +1,473 @@
+// C ABI of the fused SGP step (see include/sgp.h): handle management, argument validation, launch
+// configuration and dispatch.  All arithmetic of the method lives in the kernels.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "aux_kernels.cuh"
+#include "schedule.h"
+#include "sgp.h"
+#include "step_kernels.cuh"
+
+using sgp::ConstTable;
+using sgp::StepParams;
+
+struct sgp_handle {
+  int n = 0;
+  int64_t d = 0, ld = 0;
+  int tau = 0;
+  unsigned flags = 0;
+  int device = 0;
+  int sm_count = 0;
+  int smem_optin = 0;
+  sgp_schedule *sched = nullptr;
+  // device copy of every slot's CSR, concatenated; offsets in elements
+  int32_t *d_rowptr = nullptr;
+  int32_t *d_col = nullptr;
+  float *d_val = nullptr;
+  std::vector<int64_t> off_rowptr, off_nnz;
+  std::vector<ConstTable> const_tables;  // valid where const_ok[slot]
+  std::vector<char> const_ok;
+  float *ring_x = nullptr;   // tau * n * ld
+  float *ring_w = nullptr;   // tau * n
+  unsigned *d_words = nullptr;  // [0] ticket, [1] status
+  double *d_stats = nullptr;    // 4 doubles for sgp_check
+  int64_t opt_variant = 0, opt_tile_cols = 0, opt_ctas_per_sm = 0;
+  cudaStream_t s_h2d = nullptr, s_compute = nullptr, s_d2h = nullptr;
+  std::vector<cudaEvent_t> ev_in, ev_done;
+  int last_cuda_error = 0;
+};
+
+namespace {
+
+#define SGP_CUDA_TRY(h, expr)                                   \
+  do {                                                          \
+    cudaError_t e_ = (expr);                                    \
+    if (e_ != cudaSuccess) {                                    \
+      if (h) (h)->last_cuda_error = static_cast<int>(e_);       \
+      (void)cudaGetLastError();                                 \
+      return SGP_ERR_CUDA;                                      \
+    }                                                           \
+  } while (0)
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+inline int floor_log2(int64_t v) {
+  int l = 0;
+  while ((int64_t{1} << (l + 1)) <= v) ++l;
+  return l;
+}
+
+void free_handle(sgp_handle *h) {
+  if (h == nullptr) return;
+  cudaFree(h->d_rowptr);
+  cudaFree(h->d_col);
+  cudaFree(h->d_val);
+  cudaFree(h->ring_x);
+  cudaFree(h->ring_w);
+  cudaFree(h->d_words);
+  cudaFree(h->d_stats);
+  for (cudaEvent_t e : h->ev_in) cudaEventDestroy(e);
+  for (cudaEvent_t e : h->ev_done) cudaEventDestroy(e);
+  if (h->s_h2d) cudaStreamDestroy(h->s_h2d);
+  if (h->s_compute) cudaStreamDestroy(h->s_compute);
+  if (h->s_d2h) cudaStreamDestroy(h->s_d2h);
+  delete h->sched;
+  delete h;
+}
+
+using StepKernel = void (*)(const StepParams, const ConstTable);
+
+template <int VEC, bool HAS_M, bool NESTEROV, bool HAS_Z>
+StepKernel pick_ring(bool has_ring) {
+  return has_ring ? sgp::sgp_step_regs_kernel<VEC, HAS_M, NESTEROV, HAS_Z, true>
+                  : sgp::sgp_step_regs_kernel<VEC, HAS_M, NESTEROV, HAS_Z, false>;
+}
+template <int VEC, bool HAS_M, bool NESTEROV>
+StepKernel pick_z(bool has_z, bool has_ring) {
+  return has_z ? pick_ring<VEC, HAS_M, NESTEROV, true>(has_ring) : pick_ring<VEC, HAS_M, NESTEROV, false>(has_ring);
+}
+template <int VEC>
+StepKernel pick_update(bool has_m, bool nesterov, bool has_z, bool has_ring) {
+  if (!has_m) return pick_z<VEC, false, false>(has_z, has_ring);
+  return nesterov ? pick_z<VEC, true, true>(has_z, has_ring) : pick_z<VEC, true, false>(has_z, has_ring);
+}
+
+struct StepArgs {
+  float *X, *W, *M;
+  const float *G;
+  float *Z;
+  int64_t k;
+  float lr, momentum, wd;
+  int nesterov;
+};
+
+// One launch of the register-staged kernel over columns [c0, c1) with vector width vec.
+int launch_regs(sgp_handle *h, const StepArgs &a, int64_t c0, int64_t c1, int vec, bool update_w, cudaStream_t stream) {
+  const int64_t slot = a.k % h->sched->period();
+  const SgpStepCsr &csr = h->sched->slot(a.k);
+  StepParams p{};
+  p.X = a.X;
+  p.W = a.W;
+  p.M = a.M;
+  p.G = a.G;
+  p.Z = a.Z;
+  if (h->tau > 0) {
+    const int64_t rs = a.k % h->tau;
+    p.ring_x = h->ring_x + rs * h->n * h->ld;
+    p.ring_w = h->ring_w + rs * h->n;
+  }
+  p.ld = h->ld;
+  p.col_begin = c0;
+  p.col_end = c1;
+  p.n = h->n;
+  p.nnz = static_cast<int>(csr.col.size());
+  p.update_w = update_w ? 1 : 0;
+  p.lr = a.lr;
+  p.momentum = a.momentum;
+  p.wd = a.wd;
+  p.rowptr = h->d_rowptr + h->off_rowptr[static_cast<size_t>(slot)];
+  p.col = h->d_col + h->off_nnz[static_cast<size_t>(slot)];
+  p.val = h->d_val + h->off_nnz[static_cast<size_t>(slot)];
+  p.ticket = h->d_words;
+  p.status = h->d_words + 1;
+
+  // tile width: about kThreads * kItemsPerThread items per tile, at least 128 bytes per row segment
+  const int64_t ncols = c1 - c0;
+  const int min_tv = vec == 4 ? 8 : 32;
+  int64_t tv = int64_t{1} << floor_log2(std::max<int64_t>(1, sgp::kThreads * sgp::kItemsPerThread / h->n));
+  if (h->opt_tile_cols > 0) tv = int64_t{1} << floor_log2(std::max<int64_t>(1, h->opt_tile_cols / vec));
+  tv = std::max<int64_t>(tv, min_tv);
+  const size_t table_bytes = (static_cast<size_t>(h->n) + 1 + 2 * static_cast<size_t>(p.nnz)) * 4;
+  if (h->const_ok[static_cast<size_t>(slot)]) p.table_mode = 0;
+  else p.table_mode = table_bytes <= 40 * 1024 ? 1 : 2;
+  size_t smem = 0;
+  for (;;) {
+    smem = 2 * static_cast<size_t>(h->n) * tv * vec * 4 + 3 * static_cast<size_t>(h->n) * 4 +
+           (p.table_mode < 2 ? table_bytes : 0);
+    if (smem <= 100 * 1024 || tv <= min_tv) break;
+    tv >>= 1;
+  }
+  if (smem > static_cast<size_t>(h->smem_optin)) return SGP_ERR_ARG;
+  p.log2_tile_vecs = floor_log2(tv);
+  const int64_t tile_cols = tv * vec;
+  const int64_t ntiles = (ncols + tile_cols - 1) / tile_cols;
+  const int cps = h->opt_ctas_per_sm > 0 ? static_cast<int>(h->opt_ctas_per_sm) : 2;
+  const int64_t grid = std::min<int64_t>(ntiles, static_cast<int64_t>(h->sm_count) * cps);
+
+  const bool has_m = a.momentum != 0.0f;
+  StepKernel kern = vec == 4 ? pick_update<4>(has_m, a.nesterov != 0, a.Z != nullptr, h->tau > 0)
+                             : pick_update<1>(has_m, a.nesterov != 0, a.Z != nullptr, h->tau > 0);
+  if (smem > 48 * 1024)
+    SGP_CUDA_TRY(h, cudaFuncSetAttribute(reinterpret_cast<const void *>(kern),
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  static const ConstTable kEmptyTable{};
+  const ConstTable &ct = p.table_mode == 0 ? h->const_tables[static_cast<size_t>(slot)] : kEmptyTable;
+  kern<<<static_cast<unsigned>(grid), sgp::kThreads, smem, stream>>>(p, ct);
+  SGP_CUDA_TRY(h, cudaGetLastError());
+  return SGP_OK;
+}
+
+// The whole step over columns [c0, c1): 128-bit kernel on the aligned bulk, scalar kernel on what is left.
+int launch_step_range(sgp_handle *h, const StepArgs &a, int64_t c0, int64_t c1, bool update_w, cudaStream_t stream) {
+  const bool vec_ok = aligned16(a.X) && aligned16(a.G) && (a.M == nullptr || aligned16(a.M)) &&
+                      (a.Z == nullptr || aligned16(a.Z)) && (h->ld % 4 == 0) && (c0 % 4 == 0);
+  const int64_t vec_end = vec_ok ? c0 + ((c1 - c0) & ~int64_t{3}) : c0;
+  if (vec_end > c0) {
+    const int rc = launch_regs(h, a, c0, vec_end, 4, update_w && vec_end == c1, stream);
+    if (rc != SGP_OK) return rc;
+  }
+  if (vec_end < c1) return launch_regs(h, a, vec_end, c1, 1, update_w, stream);
+  return SGP_OK;
+}
+
+int validate_step(const sgp_handle *h, const float *X, const float *W, const float *M, const float *G, int64_t k,
+                  float momentum) {
+  if (h == nullptr || X == nullptr || W == nullptr || G == nullptr || k < 0) return SGP_ERR_ARG;
+  if (momentum != 0.0f && M == nullptr) return SGP_ERR_ARG;
+  return SGP_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int sgp_version(void) { return 100; }
+
+const char *sgp_strerror(int code) {
+  switch (code) {
+    case SGP_OK: return "ok";
+    case SGP_ERR_ARG: return "invalid argument";
+    case SGP_ERR_GRAPH: return "schedule is not a column-stochastic digraph with self-loops";
+    case SGP_ERR_CUDA: return "CUDA runtime error";
+    case SGP_ERR_ALLOC: return "allocation failed";
+    case SGP_ERR_STATE: return "call not valid for this handle";
+    case SGP_ERR_DEVICE: return "a kernel gave up a bounded wait";
+    default: return "unknown error";
+  }
+}
+
+int sgp_create(sgp_handle **out, int n, int64_t d, int64_t ld, const sgp_graph_desc *g, int tau, unsigned flags) {
+  if (out == nullptr) return SGP_ERR_ARG;
+  *out = nullptr;
+  if (n < 1 || n > SGP_MAX_NODES || d < 1 || ld < d || tau < 0 || tau > 64 || g == nullptr || flags != SGP_FLAG_NONE)
+    return SGP_ERR_ARG;
+  sgp_schedule *sched = nullptr;
+  int rc = sgp_schedule_build(&sched, n, g);
+  if (rc != SGP_OK) return rc;
+  sgp_handle *h = new (std::nothrow) sgp_handle;
+  if (h == nullptr) {
+    delete sched;
+    return SGP_ERR_ALLOC;
+  }
+  h->n = n;
+  h->d = d;
+  h->ld = ld;
+  h->tau = tau;
+  h->flags = flags;
+  h->sched = sched;
+
+  auto fail = [&](int code, cudaError_t e) {
+    const int err = static_cast<int>(e);
+    free_handle(h);
+    (void)cudaGetLastError();
+    (void)err;
+    return code;
+  };
+  cudaError_t e = cudaGetDevice(&h->device);
+  if (e != cudaSuccess) return fail(SGP_ERR_CUDA, e);
+  e = cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device);
+  if (e != cudaSuccess) return fail(SGP_ERR_CUDA, e);
+  e = cudaDeviceGetAttribute(&h->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, h->device);
+  if (e != cudaSuccess) return fail(SGP_ERR_CUDA, e);
+
+  // concatenate the slots and upload
+  std::vector<int32_t> rowptr, col;
+  std::vector<float> val;
+  const int64_t period = sched->period();
+  for (int64_t s = 0; s < period; ++s) {
+    const SgpStepCsr &c = sched->steps[static_cast<size_t>(s)];
+    h->off_rowptr.push_back(static_cast<int64_t>(rowptr.size()));
+    h->off_nnz.push_back(static_cast<int64_t>(col.size()));
+    rowptr.insert(rowptr.end(), c.rowptr.begin(), c.rowptr.end());
+    col.insert(col.end(), c.col.begin(), c.col.end());
+    val.insert(val.end(), c.val.begin(), c.val.end());
+    ConstTable ct{};
+    const bool fits = n <= sgp::kConstRows && static_cast<int>(c.col.size()) <= sgp::kConstNnz;
+    if (fits) {
+      std::copy(c.rowptr.begin(), c.rowptr.end(), ct.rowptr);
+      std::copy(c.col.begin(), c.col.end(), ct.col);
+      std::copy(c.val.begin(), c.val.end(), ct.val);
+    }
+    h->const_tables.push_back(ct);
+    h->const_ok.push_back(fits ? 1 : 0);
+  }
+  e = cudaMalloc(&h->d_rowptr, rowptr.size() * sizeof(int32_t));
+  if (e != cudaSuccess) return fail(SGP_ERR_ALLOC, e);
+  e = cudaMalloc(&h->d_col, col.size() * sizeof(int32_t));
+  if (e != cudaSuccess) return fail(SGP_ERR_ALLOC, e);
+  e = cudaMalloc(&h->d_val, val.size() * sizeof(float));
+  if (e != cudaSuccess) return fail(SGP_ERR_ALLOC, e);
+  e = cudaMalloc(&h->d_words, 2 * sizeof(unsigned));
+  if (e != cudaSuccess) return fail(SGP_ERR_ALLOC, e);
+  e = cudaMalloc(&h->d_stats, 4 * sizeof(double));
+  if (e != cudaSuccess) return fail(SGP_ERR_ALLOC, e);
+  if (tau > 0) {
+    e = cudaMalloc(&h->ring_x, static_cast<size_t>(tau) * n * ld * sizeof(float));
+    if (e != cudaSuccess) return fail(SGP_ERR_ALLOC, e);
+    e = cudaMalloc(&h->ring_w, static_cast<size_t>(tau) * n * sizeof(float));
+    if (e != cudaSuccess) return fail(SGP_ERR_ALLOC, e);
+    e = cudaMemset(h->ring_x, 0, static_cast<size_t>(tau) * n * ld * sizeof(float));
+    if (e != cudaSuccess) return fail(SGP_ERR_CUDA, e);
+    e = cudaMemset(h->ring_w, 0, static_cast<size_t>(tau) * n * sizeof(float));
+    if (e != cudaSuccess) return fail(SGP_ERR_CUDA, e);
+  }
+  e = cudaMemcpy(h->d_rowptr, rowptr.data(), rowptr.size() * sizeof(int32_t), cudaMemcpyHostToDevice);
+  if (e != cudaSuccess) return fail(SGP_ERR_CUDA, e);
+  e = cudaMemcpy(h->d_col, col.data(), col.size() * sizeof(int32_t), cudaMemcpyHostToDevice);
+  if (e != cudaSuccess) return fail(SGP_ERR_CUDA, e);
+  e = cudaMemcpy(h->d_val, val.data(), val.size() * sizeof(float), cudaMemcpyHostToDevice);
+  if (e != cudaSuccess) return fail(SGP_ERR_CUDA, e);
+  e = cudaMemset(h->d_words, 0, 2 * sizeof(unsigned));
+  if (e != cudaSuccess) return fail(SGP_ERR_CUDA, e);
+  e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return fail(SGP_ERR_CUDA, e);
+  *out = h;
+  return SGP_OK;
+}
+
+int sgp_destroy(sgp_handle *h) {
+  if (h == nullptr) return SGP_OK;
+  (void)cudaDeviceSynchronize();
+  free_handle(h);
+  return SGP_OK;
+}
+
+int sgp_get_schedule(const sgp_handle *h, const sgp_schedule **s) {
+  if (h == nullptr || s == nullptr) return SGP_ERR_ARG;
+  *s = h->sched;
+  return SGP_OK;
+}
+
+int sgp_step(sgp_handle *h, float *d_X, float *d_W, float *d_M, const float *d_G, float *d_Z, int64_t k, float lr,
+             float momentum, float weight_decay, int nesterov, void *stream) {
+  const int rc = validate_step(h, d_X, d_W, d_M, d_G, k, momentum);
+  if (rc != SGP_OK) return rc;
+  const StepArgs a{d_X, d_W, momentum != 0.0f ? d_M : nullptr, d_G, d_Z, k, lr, momentum, weight_decay, nesterov};
+  return launch_step_range(h, a, 0, h->d, true, static_cast<cudaStream_t>(stream));
+}
+
+int sgp_debias(sgp_handle *h, const float *d_X, const float *d_W, float *d_Z, void *stream) {
+  if (h == nullptr || d_X == nullptr || d_W == nullptr || d_Z == nullptr) return SGP_ERR_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const bool vec_ok = aligned16(d_X) && aligned16(d_Z) && (h->ld % 4 == 0);
+  const int64_t work = vec_ok ? (h->d + 3) / 4 : h->d;
+  const int64_t per_row = std::max<int64_t>(1, (static_cast<int64_t>(h->sm_count) * 8 + h->n - 1) / h->n);
+  const unsigned gx = static_cast<unsigned>(std::max<int64_t>(1, std::min<int64_t>((work + 255) / 256, per_row)));
+  const dim3 grid(gx, static_cast<unsigned>(h->n));
+  if (vec_ok) sgp::sgp_debias_kernel<4><<<grid, 256, 0, st>>>(d_X, d_W, d_Z, h->d, h->ld);
+  else sgp::sgp_debias_kernel<1><<<grid, 256, 0, st>>>(d_X, d_W, d_Z, h->d, h->ld);
+  SGP_CUDA_TRY(h, cudaGetLastError());
+  return SGP_OK;
+}
+
+int sgp_step_host(sgp_handle *h, float *d_X, float *d_W, float *d_M, const float *h_G, float *h_Z, float *d_G,
+                  float *d_Z, int64_t k, float lr, float momentum, float weight_decay, int nesterov,
+                  int64_t chunk_cols) {
+  int rc = validate_step(h, d_X, d_W, d_M, d_G, k, momentum);
+  if (rc != SGP_OK) return rc;
+  if (h_G == nullptr || (h_Z != nullptr && d_Z == nullptr)) return SGP_ERR_ARG;
+  if (h->s_h2d == nullptr) {
+    SGP_CUDA_TRY(h, cudaStreamCreateWithFlags(&h->s_h2d, cudaStreamNonBlocking));
+    SGP_CUDA_TRY(h, cudaStreamCreateWithFlags(&h->s_compute, cudaStreamNonBlocking));
+    SGP_CUDA_TRY(h, cudaStreamCreateWithFlags(&h->s_d2h, cudaStreamNonBlocking));
+  }
+  // default chunk: about 64 MB of gradient per chunk, a multiple of 1024 columns
+  if (chunk_cols <= 0) chunk_cols = std::max<int64_t>(1024, (int64_t{64} << 20) / (4 * h->n) / 1024 * 1024);
+  chunk_cols = (chunk_cols + 3) / 4 * 4;
+  const int64_t nchunks = (h->d + chunk_cols - 1) / chunk_cols;
+  while (static_cast<int64_t>(h->ev_in.size()) < nchunks) {
+    cudaEvent_t a = nullptr, b = nullptr;
+    SGP_CUDA_TRY(h, cudaEventCreateWithFlags(&a, cudaEventDisableTiming));
+    h->ev_in.push_back(a);
+    SGP_CUDA_TRY(h, cudaEventCreateWithFlags(&b, cudaEventDisableTiming));
+    h->ev_done.push_back(b);
+  }
+  // earlier work of the caller on the legacy/default stream must be visible
+  SGP_CUDA_TRY(h, cudaDeviceSynchronize());
+  const StepArgs a{d_X, d_W, momentum != 0.0f ? d_M : nullptr, d_G, h_Z != nullptr ? d_Z : nullptr,
+                   k, lr, momentum, weight_decay, nesterov};
+  const size_t pitch = static_cast<size_t>(h->ld) * sizeof(float);
+  for (int64_t c = 0; c < nchunks; ++c) {
+    const int64_t c0 = c * chunk_cols, c1 = std::min(h->d, c0 + chunk_cols);
+    const size_t width = static_cast<size_t>(c1 - c0) * sizeof(float);
+    SGP_CUDA_TRY(h, cudaMemcpy2DAsync(d_G + c0, pitch, h_G + c0, pitch, width, static_cast<size_t>(h->n),
+                                      cudaMemcpyHostToDevice, h->s_h2d));
+    SGP_CUDA_TRY(h, cudaEventRecord(h->ev_in[static_cast<size_t>(c)], h->s_h2d));
+    SGP_CUDA_TRY(h, cudaStreamWaitEvent(h->s_compute, h->ev_in[static_cast<size_t>(c)], 0));
+    rc = launch_step_range(h, a, c0, c1, c == nchunks - 1, h->s_compute);
+    if (rc != SGP_OK) return rc;
+    if (h_Z != nullptr) {
+      SGP_CUDA_TRY(h, cudaEventRecord(h->ev_done[static_cast<size_t>(c)], h->s_compute));
+      SGP_CUDA_TRY(h, cudaStreamWaitEvent(h->s_d2h, h->ev_done[static_cast<size_t>(c)], 0));
+      SGP_CUDA_TRY(h, cudaMemcpy2DAsync(h_Z + c0, pitch, d_Z + c0, pitch, width, static_cast<size_t>(h->n),
+                                        cudaMemcpyDeviceToHost, h->s_d2h));
+    }
+  }
+  SGP_CUDA_TRY(h, cudaStreamSynchronize(h->s_h2d));
+  SGP_CUDA_TRY(h, cudaStreamSynchronize(h->s_compute));
+  SGP_CUDA_TRY(h, cudaStreamSynchronize(h->s_d2h));
+  return SGP_OK;
+}
+
+int sgp_reset(sgp_handle *h, void *stream) {
+  if (h == nullptr) return SGP_ERR_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (h->tau > 0) {
+    SGP_CUDA_TRY(h, cudaMemsetAsync(h->ring_x, 0, static_cast<size_t>(h->tau) * h->n * h->ld * sizeof(float), st));
+    SGP_CUDA_TRY(h, cudaMemsetAsync(h->ring_w, 0, static_cast<size_t>(h->tau) * h->n * sizeof(float), st));
+  }
+  SGP_CUDA_TRY(h, cudaMemsetAsync(h->d_words, 0, 2 * sizeof(unsigned), st));
+  return SGP_OK;
+}
+
+int sgp_ring_export(sgp_handle *h, float *d_ring_x, float *d_ring_w, void *stream) {
+  if (h == nullptr || d_ring_x == nullptr || d_ring_w == nullptr) return SGP_ERR_ARG;
+  if (h->tau == 0) return SGP_ERR_STATE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  SGP_CUDA_TRY(h, cudaMemcpyAsync(d_ring_x, h->ring_x, static_cast<size_t>(h->tau) * h->n * h->ld * sizeof(float),
+                                  cudaMemcpyDeviceToDevice, st));
+  SGP_CUDA_TRY(h, cudaMemcpyAsync(d_ring_w, h->ring_w, static_cast<size_t>(h->tau) * h->n * sizeof(float),
+                                  cudaMemcpyDeviceToDevice, st));
+  return SGP_OK;
+}
+
+int sgp_ring_import(sgp_handle *h, const float *d_ring_x, const float *d_ring_w, void *stream) {
+  if (h == nullptr || d_ring_x == nullptr || d_ring_w == nullptr) return SGP_ERR_ARG;
+  if (h->tau == 0) return SGP_ERR_STATE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  SGP_CUDA_TRY(h, cudaMemcpyAsync(h->ring_x, d_ring_x, static_cast<size_t>(h->tau) * h->n * h->ld * sizeof(float),
+                                  cudaMemcpyDeviceToDevice, st));
+  SGP_CUDA_TRY(h, cudaMemcpyAsync(h->ring_w, d_ring_w, static_cast<size_t>(h->tau) * h->n * sizeof(float),
+                                  cudaMemcpyDeviceToDevice, st));
+  return SGP_OK;
+}
+
+int sgp_check(sgp_handle *h, const float *d_X, const float *d_W, double *h_stats, void *stream) {
+  if (h == nullptr || d_X == nullptr || d_W == nullptr || h_stats == nullptr) return SGP_ERR_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  SGP_CUDA_TRY(h, cudaMemsetAsync(h->d_stats, 0, 4 * sizeof(double), st));
+  const unsigned grid = static_cast<unsigned>(h->sm_count * 8);
+  sgp::sgp_scan_kernel<<<grid, 256, 0, st>>>(d_X, h->n, h->d, h->ld, h->d_stats);
+  if (h->tau > 0) sgp::sgp_scan_kernel<<<grid, 256, 0, st>>>(h->ring_x, h->tau * h->n, h->d, h->ld, h->d_stats);
+  sgp::sgp_weight_scan_kernel<<<1, 256, 0, st>>>(d_W, h->n, h->ring_w, h->tau * h->n, h->d_stats);
+  SGP_CUDA_TRY(h, cudaGetLastError());
+  double tmp[4];
+  SGP_CUDA_TRY(h, cudaMemcpyAsync(tmp, h->d_stats, sizeof(tmp), cudaMemcpyDeviceToHost, st));
+  SGP_CUDA_TRY(h, cudaStreamSynchronize(st));
+  h_stats[0] = tmp[2];
+  h_stats[1] = tmp[3];
+  h_stats[2] = tmp[1];
+  h_stats[3] = tmp[0];
+  return SGP_OK;
+}
+
+int sgp_set_option(sgp_handle *h, const char *key, int64_t value) {
+  if (h == nullptr || key == nullptr || value < 0) return SGP_ERR_ARG;
+  if (std::strcmp(key, "variant") == 0) {
+    if (value > 2) return SGP_ERR_ARG;
+    h->opt_variant = value;
+  } else if (std::strcmp(key, "tile_cols") == 0) {
+    if (value % 4 != 0 || value > 4096) return SGP_ERR_ARG;
+    h->opt_tile_cols = value;
+  } else if (std::strcmp(key, "ctas_per_sm") == 0) {
+    if (value > 16) return SGP_ERR_ARG;
+    h->opt_ctas_per_sm = value;
+  } else {
+    return SGP_ERR_ARG;
+  }
+  return SGP_OK;
+}
+
+int sgp_get_option(const sgp_handle *h, const char *key, int64_t *value) {
+  if (h == nullptr || key == nullptr || value == nullptr) return SGP_ERR_ARG;
+  if (std::strcmp(key, "variant") == 0) *value = h->opt_variant;
+  else if (std::strcmp(key, "tile_cols") == 0) *value = h->opt_tile_cols;
+  else if (std::strcmp(key, "ctas_per_sm") == 0) *value = h->opt_ctas_per_sm;
+  else return SGP_ERR_ARG;
+  return SGP_OK;
+}
+
+int sgp_device_status(sgp_handle *h, unsigned *status) {
+  if (h == nullptr || status == nullptr) return SGP_ERR_ARG;
+  SGP_CUDA_TRY(h, cudaDeviceSynchronize());
+  SGP_CUDA_TRY(h, cudaMemcpy(status, h->d_words + 1, sizeof(unsigned), cudaMemcpyDeviceToHost));
+  return SGP_OK;
+}
+
+int sgp_last_cuda_error(const sgp_handle *h) { return h == nullptr ? 0 : h->last_cuda_error; }
+
+}  // extern "C"

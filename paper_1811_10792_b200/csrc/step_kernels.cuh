@@ -1,0 +1,268 @@
+// Fused SGP step kernels for sm_100a.
+//
+// One persistent CTA owns, tile after tile, ALL n rows of a block of columns: the mix of Alg. 1
+// line 6 couples rows (nodes) but never columns, so a CTA that holds x^(k+1/2) of every node for
+// its columns can finish the whole iteration -- local update (Alg. 3 lines 4-5), gather-mix,
+// delayed-message ring (Alg. 2), de-bias (Alg. 1 line 8) -- with one read and one write of each
+// array and no inter-CTA dependency (no grid sync, no device-side wait on another CTA).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace sgp {
+
+constexpr int kThreads = 256;       // threads per CTA of the register-staged kernel
+constexpr int kItemsPerThread = 4;  // (row, vector-column) items a thread keeps in flight per batch
+
+// Mixing table of one step small enough to travel as a kernel argument (constant bank).
+constexpr int kConstRows = 64;
+constexpr int kConstNnz = 320;
+struct ConstTable {
+  int32_t rowptr[kConstRows + 1];
+  int32_t col[kConstNnz];
+  float val[kConstNnz];
+};
+
+struct StepParams {
+  float *X;
+  float *W;
+  float *M;        // may be null when momentum == 0
+  const float *G;
+  float *Z;        // may be null
+  float *ring_x;   // this step's ring slot (n x ld) or null when tau == 0
+  float *ring_w;   // this step's weight-ring slot (n) or null
+  int64_t ld;
+  int64_t col_begin;  // first column this launch processes
+  int64_t col_end;    // one past the last column
+  int n;
+  int nnz;
+  int log2_tile_vecs;  // tile width in vectors (power of two)
+  int update_w;        // 1: this launch also commits W (and the weight ring) for the step
+  int table_mode;      // 0: copy table from the kernel argument, 1: copy from global, 2: read global in place
+  float lr, momentum, wd;
+  const int32_t *rowptr;  // global copy of the step's CSR (always valid)
+  const int32_t *col;
+  const float *val;
+  unsigned *ticket;  // arrival counter for the last-CTA-commits-W protocol (self-resetting)
+  unsigned *status;  // device status word
+};
+
+template <int VEC> struct VecT;
+template <> struct VecT<4> { using type = float4; };
+template <> struct VecT<1> { using type = float; };
+
+__device__ __forceinline__ float4 ld_stream(const float4 *p) { return __ldcs(p); }
+__device__ __forceinline__ float ld_stream(const float *p) { return __ldcs(p); }
+__device__ __forceinline__ void st_stream(float4 *p, float4 v) { __stcs(p, v); }
+__device__ __forceinline__ void st_stream(float *p, float v) { __stcs(p, v); }
+
+__device__ __forceinline__ float4 vfma(float a, float4 b, float4 c) {
+  return make_float4(fmaf(a, b.x, c.x), fmaf(a, b.y, c.y), fmaf(a, b.z, c.z), fmaf(a, b.w, c.w));
+}
+__device__ __forceinline__ float vfma(float a, float b, float c) { return fmaf(a, b, c); }
+__device__ __forceinline__ float4 vmul(float a, float4 b) { return make_float4(a * b.x, a * b.y, a * b.z, a * b.w); }
+__device__ __forceinline__ float vmul(float a, float b) { return a * b; }
+__device__ __forceinline__ float4 vadd(float4 a, float4 b) { return make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w); }
+__device__ __forceinline__ float vadd(float a, float b) { return a + b; }
+template <typename V> __device__ __forceinline__ V vzero();
+template <> __device__ __forceinline__ float4 vzero<float4>() { return make_float4(0.f, 0.f, 0.f, 0.f); }
+template <> __device__ __forceinline__ float vzero<float>() { return 0.f; }
+
+// Local update of one element group: returns h = x^(k+1/2) and the new momentum (Alg. 3 lines 4-5;
+// Alg. 1 line 4 when there is no momentum).  Weight decay adds wd * x to the gradient.
+template <bool HAS_M, bool NESTEROV, typename V>
+__device__ __forceinline__ V local_update(V x, V g, V &u, float lr, float momentum, float wd) {
+  V gt = vfma(wd, x, g);
+  V s;
+  if (HAS_M) {
+    u = vfma(momentum, u, gt);
+    s = NESTEROV ? vfma(momentum, u, gt) : u;
+  } else {
+    s = gt;
+  }
+  return vfma(-lr, s, x);
+}
+
+// Shared-memory carve-up (dynamic): [H tile: tile_items vectors][w_old n][rw_in n][inv_w n][p_self n]
+// then the CSR copy when table_mode < 2.
+struct CtaTables {
+  const int32_t *rowptr;
+  const int32_t *col;
+  const float *val;
+  float *inv_w;
+};
+
+// Per-CTA prologue shared by the step kernels: stage the step's CSR, mix the push-sum weights
+// (Alg. 1 line 7 / Alg. 2 lines 8, 22) and, when this launch owns the commit, let the LAST CTA to
+// arrive write W and the weight ring back.  Every CTA takes its ticket only after its own reads of
+// the old W have completed, so the committing CTA knows no reader is left; nobody waits for anybody.
+template <bool HAS_RING>
+__device__ __forceinline__ CtaTables cta_prologue(const StepParams &p, const ConstTable &ct, float *scratch, int nthreads) {
+  const int n = p.n;
+  float *w_old = scratch;
+  float *rw_in = scratch + n;
+  float *inv_w = scratch + 2 * n;
+  int32_t *s_rowptr = reinterpret_cast<int32_t *>(scratch + 3 * n);
+  int32_t *s_col = s_rowptr + (n + 1);
+  float *s_val = reinterpret_cast<float *>(s_col + p.nnz);
+  __shared__ int s_is_last;
+
+  CtaTables t;
+  t.inv_w = inv_w;
+  if (p.table_mode == 2) {
+    t.rowptr = p.rowptr;
+    t.col = p.col;
+    t.val = p.val;
+  } else {
+    const int32_t *src_rowptr = p.table_mode == 0 ? ct.rowptr : p.rowptr;
+    const int32_t *src_col = p.table_mode == 0 ? ct.col : p.col;
+    const float *src_val = p.table_mode == 0 ? ct.val : p.val;
+    for (int i = threadIdx.x; i <= n; i += nthreads) s_rowptr[i] = src_rowptr[i];
+    for (int e = threadIdx.x; e < p.nnz; e += nthreads) {
+      s_col[e] = src_col[e];
+      s_val[e] = src_val[e];
+    }
+    t.rowptr = s_rowptr;
+    t.col = s_col;
+    t.val = s_val;
+  }
+  for (int i = threadIdx.x; i < n; i += nthreads) {
+    w_old[i] = p.W[i];
+    if (HAS_RING) rw_in[i] = p.ring_w[i];
+  }
+  __syncthreads();
+  if (p.update_w && threadIdx.x == 0) {
+    __threadfence();
+    const unsigned ticket = atomicAdd(p.ticket, 1u);
+    s_is_last = (ticket == gridDim.x - 1) ? 1 : 0;
+  }
+  __syncthreads();
+  const bool commit = p.update_w && s_is_last;
+  for (int i = threadIdx.x; i < n; i += nthreads) {
+    float acc = 0.f, off = 0.f;
+    for (int e = t.rowptr[i]; e < t.rowptr[i + 1]; ++e) {
+      const int j = t.col[e];
+      const float pv = t.val[e];
+      if (HAS_RING && j != i) off = fmaf(pv, w_old[j], off);
+      else acc = fmaf(pv, w_old[j], acc);
+    }
+    if (HAS_RING) acc += rw_in[i];
+    inv_w[i] = 1.0f / acc;
+    if (commit) {
+      p.W[i] = acc;
+      if (HAS_RING) p.ring_w[i] = off;
+    }
+  }
+  if (commit && threadIdx.x == 0) *p.ticket = 0u;  // ready for the next launch
+  __syncthreads();
+  return t;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Register-staged kernel: every thread keeps kItemsPerThread (row, vector-column) items in flight,
+// writes x^(k+1/2) into a shared tile, one barrier, then gathers its receivers' rows from the tile.
+// The tile is double-buffered so one barrier per batch suffices.
+// ------------------------------------------------------------------------------------------------
+template <int VEC, bool HAS_M, bool NESTEROV, bool HAS_Z, bool HAS_RING>
+__global__ void __launch_bounds__(kThreads, 2)
+sgp_step_regs_kernel(const __grid_constant__ StepParams p, const __grid_constant__ ConstTable ct) {
+  using V = typename VecT<VEC>::type;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int n = p.n;
+  const int tv = 1 << p.log2_tile_vecs;
+  const int tile_items = n * tv;
+  V *H0 = reinterpret_cast<V *>(smem_raw);
+  V *H1 = H0 + tile_items;
+  float *scratch = reinterpret_cast<float *>(H1 + tile_items);
+  const CtaTables tab = cta_prologue<HAS_RING>(p, ct, scratch, kThreads);
+
+  const int64_t ld = p.ld;
+  const int64_t ncols = p.col_end - p.col_begin;
+  const int64_t tile_cols = static_cast<int64_t>(tv) * VEC;
+  const int64_t ntiles = (ncols + tile_cols - 1) / tile_cols;
+  const float lr = p.lr, momentum = p.momentum, wd = p.wd;
+  int buf = 0;
+
+  for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+    const int64_t col0 = p.col_begin + tile * tile_cols;
+    V *H = buf ? H1 : H0;
+    // ---- phase 1: local update, all batches of this tile
+    for (int base = 0; base < tile_items; base += kThreads * kItemsPerThread) {
+      V x[kItemsPerThread], g[kItemsPerThread], u[kItemsPerThread];
+      bool ok[kItemsPerThread];
+      int64_t off[kItemsPerThread];
+#pragma unroll
+      for (int q = 0; q < kItemsPerThread; ++q) {
+        const int item = base + q * kThreads + threadIdx.x;
+        const int row = item >> p.log2_tile_vecs;
+        const int c = item & (tv - 1);
+        const int64_t col = col0 + static_cast<int64_t>(c) * VEC;
+        ok[q] = (item < tile_items) && (col < p.col_end);
+        off[q] = static_cast<int64_t>(row) * ld + col;
+      }
+#pragma unroll
+      for (int q = 0; q < kItemsPerThread; ++q) {
+        if (ok[q]) {
+          x[q] = ld_stream(reinterpret_cast<const V *>(p.X + off[q]));
+          g[q] = ld_stream(reinterpret_cast<const V *>(p.G + off[q]));
+          if (HAS_M) u[q] = ld_stream(reinterpret_cast<const V *>(p.M + off[q]));
+        }
+      }
+#pragma unroll
+      for (int q = 0; q < kItemsPerThread; ++q) {
+        const int item = base + q * kThreads + threadIdx.x;
+        if (ok[q]) {
+          const V h = local_update<HAS_M, NESTEROV, V>(x[q], g[q], u[q], lr, momentum, wd);
+          if (HAS_M) st_stream(reinterpret_cast<V *>(p.M + off[q]), u[q]);
+          H[item] = h;
+        } else if (item < tile_items) {
+          H[item] = vzero<V>();
+        }
+      }
+    }
+    __syncthreads();
+    // ---- phase 2: gather-mix over the step's in-neighbour lists, ring exchange, de-bias
+    for (int base = 0; base < tile_items; base += kThreads * kItemsPerThread) {
+      V ring_in[kItemsPerThread];
+      if (HAS_RING) {
+#pragma unroll
+        for (int q = 0; q < kItemsPerThread; ++q) {
+          const int item = base + q * kThreads + threadIdx.x;
+          const int row = item >> p.log2_tile_vecs;
+          const int c = item & (tv - 1);
+          const int64_t col = col0 + static_cast<int64_t>(c) * VEC;
+          if (item < tile_items && col < p.col_end)
+            ring_in[q] = ld_stream(reinterpret_cast<const V *>(p.ring_x + static_cast<int64_t>(row) * ld + col));
+        }
+      }
+#pragma unroll
+      for (int q = 0; q < kItemsPerThread; ++q) {
+        const int item = base + q * kThreads + threadIdx.x;
+        const int row = item >> p.log2_tile_vecs;
+        const int c = item & (tv - 1);
+        const int64_t col = col0 + static_cast<int64_t>(c) * VEC;
+        if (item < tile_items && col < p.col_end) {
+          const int64_t o = static_cast<int64_t>(row) * ld + col;
+          V acc = vzero<V>(), offd = vzero<V>();
+          const int e1 = tab.rowptr[row + 1];
+          for (int e = tab.rowptr[row]; e < e1; ++e) {
+            const int j = tab.col[e];
+            const float pv = tab.val[e];
+            const V hj = H[(j << p.log2_tile_vecs) + c];
+            if (HAS_RING && j != row) offd = vfma(pv, hj, offd);
+            else acc = vfma(pv, hj, acc);
+          }
+          if (HAS_RING) {
+            acc = vadd(acc, ring_in[q]);
+            st_stream(reinterpret_cast<V *>(p.ring_x + o), offd);
+          }
+          st_stream(reinterpret_cast<V *>(p.X + o), acc);
+          if (HAS_Z) st_stream(reinterpret_cast<V *>(p.Z + o), vmul(tab.inv_w[row], acc));
+        }
+      }
+    }
+    buf ^= 1;
+  }
+}
+
+}  // namespace sgp

@@ -1,0 +1,327 @@
+"""GPU parity: the fused CUDA step (through the C ABI) against the float64 oracle, element by element,
+on the same seeded inputs.  Sizes span several column tiles and a ragged tail; the w != 1 cases
+(irregular graphs, delayed messages) are included because regular graphs cannot detect a broken
+weight path."""
+import numpy as np
+import pytest
+import torch
+
+from conftest import read_golden
+from parity_util import REL_TOL, assert_close, graph_desc, oracle_P_of_k, run_oracle
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_1811_10792_b200 import build
+    build.build()
+    from paper_1811_10792_b200 import binding as b
+    return b
+
+
+@pytest.fixture(scope="module")
+def inputs():
+    from paper_1811_10792_b200 import inputs as i
+    return i
+
+
+def _run_gpu(binding, inputs, w, K=None, ld=None, write_z=True, options=None, graph=None, x0=None, offset=0):
+    """Runs K fused steps on the GPU; returns (x0, grads, X, W, M, Z, handle-free ring copies)."""
+    K = w.K if K is None else K
+    n, d = w.n, w.d
+    ld = d if ld is None else ld
+    pad = float("nan")
+    def alloc():
+        buf = torch.full((n * ld + offset + 8,), pad, dtype=torch.float32, device=DEV)
+        return buf, buf[offset:offset + n * ld].view(n, ld)[:, :d]
+    Xb, X = alloc()
+    Mb, M = alloc()
+    Gb, G = alloc()
+    Zb, Z = alloc()
+    X.copy_(inputs.initial_x(w, device=DEV) if x0 is None else torch.as_tensor(x0, dtype=torch.float32, device=DEV))
+    M.zero_()
+    W = torch.ones(n, dtype=torch.float32, device=DEV)
+    x0_bits = X.cpu().numpy().copy()
+    grads = []
+    ring = None
+    with binding.Sgp(n, d, graph_desc(w, binding) if graph is None else graph, tau=w.tau, ld=ld) as h:
+        for key, val in (options or {}).items():
+            h.set_option(key, val)
+        for k in range(K):
+            inputs.gradient(w, k, G)
+            grads.append(G.cpu().numpy().copy())
+            h.step(X, W, M if w.momentum != 0.0 else None, G, Z if write_z else None, k, w.lr, w.momentum,
+                   w.weight_decay, w.nesterov)
+        torch.cuda.synchronize()
+        assert h.device_status() == 0
+        stats = h.check(X, W)
+        if w.tau > 0:
+            rx = torch.empty((w.tau, n, ld), dtype=torch.float32, device=DEV)
+            rw = torch.empty((w.tau, n), dtype=torch.float32, device=DEV)
+            h.ring_export(rx, rw)
+            torch.cuda.synchronize()
+            ring = (rx[:, :, :d].cpu().numpy(), rw.cpu().numpy())
+    # padding between rows and around the arrays must be untouched (NaN sentinels)
+    for name, buf in (("X", Xb), ("M", Mb), ("Z", Zb)):
+        full = buf.cpu().numpy()
+        mask = np.ones(full.shape, dtype=bool)
+        body = mask[offset:offset + n * ld].reshape(n, ld)
+        body[:, :d] = False
+        assert np.all(np.isnan(full[mask])), f"{name}: padding was overwritten"
+    return dict(x0=x0_bits, grads=grads, X=X.cpu().numpy(), W=W.cpu().numpy(), M=M.cpu().numpy(),
+                Z=Z.cpu().numpy(), ring=ring, stats=stats)
+
+
+def _compare(w, out, K=None, write_z=True, P_of_k=None):
+    from oracle import sgp as osgp
+    K = w.K if K is None else K
+    if P_of_k is None:
+        st = run_oracle(w, out["x0"], out["grads"], K=K)
+    else:
+        st = osgp.sgp_run(out["x0"].astype(np.float64), K, P_of_k, lambda k, z: out["grads"][k].astype(np.float64),
+                          w.lr, momentum=w.momentum, nesterov=w.nesterov, weight_decay=w.weight_decay, tau=w.tau)
+    assert_close("X", out["X"], st.x)
+    assert_close("W", out["W"], st.w)
+    if w.momentum != 0.0:
+        assert_close("M", out["M"], st.u)
+    if write_z:
+        assert_close("Z", out["Z"], st.z)
+    if w.tau > 0:
+        # ring slot s holds the message written at the last step k with k mod tau == s
+        ring_x, ring_w = out["ring"]
+        msgs_x, msgs_w = list(st.transit_x), list(st.transit_w)      # oldest first: sent at K-tau .. K-1
+        for age, (mx, mw) in enumerate(zip(msgs_x, msgs_w)):
+            k_sent = K - w.tau + age
+            assert_close(f"ring_x[{k_sent % w.tau}]", ring_x[k_sent % w.tau], mx)
+            assert_close(f"ring_w[{k_sent % w.tau}]", ring_w[k_sent % w.tau], mw)
+    # invariants from the GPU's own check kernel
+    sum_w, min_w, nonfinite, _ = out["stats"]
+    assert abs(sum_w - w.n) <= 1e-4 * w.n and min_w > 0 and nonfinite == 0
+    return st
+
+
+# ------------------------------------------------------------------ the BASELINE configurations, oracle-sized
+def test_config1_tiny_closed_loop(binding, inputs):
+    """n=8, d=4096, K=100, one-peer graph, Nesterov; g = z - c + noise computed from each side's OWN z."""
+    from oracle import sgp as osgp
+    w = inputs.WORKLOADS["tiny"]
+    n, d, K = w.n, w.d, w.K
+    c = inputs.normal(n, d, seed=w.seed, stream=inputs.STREAM_TARGET, step=0, std=1.0, device=DEV)
+    noise = [inputs.normal(n, d, seed=w.seed, stream=inputs.STREAM_NOISE, step=k, std=0.1, device=DEV) for k in range(K)]
+    X = torch.zeros((n, d), device=DEV)
+    W = torch.ones(n, device=DEV)
+    M = torch.zeros_like(X)
+    Z = X.clone()
+    with binding.Sgp(n, d, binding.GraphDesc.exp_peers(1)) as h:
+        for k in range(K):
+            G = Z - c + noise[k]                      # harness arithmetic (gradient oracle), not the SGP path
+            h.step(X, W, M, G, Z, k, w.lr, w.momentum, 0.0, True)
+        torch.cuda.synchronize()
+    c64 = c.cpu().numpy().astype(np.float64)
+    nz = [t.cpu().numpy().astype(np.float64) for t in noise]
+    st = osgp.sgp_run(np.zeros((n, d)), K, oracle_P_of_k(w), lambda k, z: z - c64 + nz[k], w.lr, momentum=w.momentum,
+                      nesterov=True)
+    assert_close("X", X.cpu().numpy(), st.x)
+    assert_close("Z", Z.cpu().numpy(), st.z)
+    assert_close("M", M.cpu().numpy(), st.u)
+    assert np.array_equal(W.cpu().numpy(), np.ones(n, dtype=np.float32))
+    # the run really optimises: consensus around mean(c)
+    assert np.abs(st.z.mean(axis=0) - c64.mean(axis=0)).max() < 0.2
+
+
+@pytest.mark.parametrize("d", [8200, 128 * 37, 1000])
+def test_config2_resnet_recipe_scaled(binding, inputs, d):
+    w = inputs.WORKLOADS["resnet50"].scaled(d)
+    out = _run_gpu(binding, inputs, w)
+    st = _compare(w, out)
+    assert np.array_equal(out["W"], np.ones(w.n, dtype=np.float32))      # regular graph
+
+
+@pytest.mark.parametrize("d", [256 * 9 + 12, 5000])
+def test_config3_transformer_recipe_scaled(binding, inputs, d):
+    w = inputs.WORKLOADS["transformer"].scaled(d)
+    out = _run_gpu(binding, inputs, w)
+    _compare(w, out)
+    assert np.all(np.isnan(out["M"]) | (out["M"] == 0))                  # plain SGD never touches M
+
+
+@pytest.mark.parametrize("tau", [1, 2, 3])
+def test_config4_overlap_scaled(binding, inputs, tau):
+    import dataclasses
+    w = dataclasses.replace(inputs.WORKLOADS["resnet50_osgp1"].scaled(4104, K=20), tau=tau)
+    out = _run_gpu(binding, inputs, w)
+    st = _compare(w, out)
+    assert abs(out["W"][0] - 1.0) > 0.2                                  # mass in transit: w != 1
+
+
+@pytest.mark.parametrize("n", [4, 16, 64, 256])
+@pytest.mark.parametrize("d", [10_000, 1029])
+def test_config5_sweep_points(binding, inputs, n, d):
+    w = inputs.sweep_workload(n, d)
+    out = _run_gpu(binding, inputs, w)
+    _compare(w, out)
+    assert np.ptp(out["W"]) > 1e-3                                       # irregular graph: weights differ
+
+
+@pytest.mark.parametrize("tau", [0, 2])
+def test_random_graph_with_delay_and_weight_decay(binding, inputs, tau):
+    import dataclasses
+    w = dataclasses.replace(inputs.sweep_workload(16, 3000), tau=tau, weight_decay=1e-2, K=13)
+    out = _run_gpu(binding, inputs, w)
+    _compare(w, out)
+
+
+# ------------------------------------------------------------------ degenerate and ragged shapes
+@pytest.mark.parametrize("n", [1, 2, 3, 5, 8])
+@pytest.mark.parametrize("d", [1, 3, 4, 5, 127, 128, 129])
+def test_small_shapes(binding, inputs, n, d):
+    w = inputs.Workload("small", n=n, d=d, K=5, graph="exp", peers=1, lr=0.1, momentum=0.9, weight_decay=1e-3)
+    out = _run_gpu(binding, inputs, w)
+    _compare(w, out)
+
+
+@pytest.mark.parametrize("ld_extra,offset", [(0, 0), (4, 0), (3, 0), (0, 1), (8, 4)])
+def test_pitch_and_alignment_paths(binding, inputs, ld_extra, offset):
+    """ld > d, ld not a multiple of 4 and pointers off 16-byte alignment: vector and scalar paths, same numbers."""
+    w = inputs.sweep_workload(16, 2052)
+    out = _run_gpu(binding, inputs, w, ld=w.d + ld_extra, offset=offset)
+    _compare(w, out)
+
+
+def test_without_z_and_heavy_ball(binding, inputs):
+    import dataclasses
+    w = dataclasses.replace(inputs.sweep_workload(16, 2500), nesterov=False)
+    out = _run_gpu(binding, inputs, w, write_z=False)
+    _compare(w, out, write_z=False)
+    assert np.all(np.isnan(out["Z"]))                                    # Z = NULL: never written
+
+
+def test_complete_graph_is_parallel_sgd(binding, inputs):
+    """All-to-all mixing with n = 256 (table read from global memory in place); identical init => AllReduce SGD."""
+    w = inputs.Workload("complete", n=256, d=520, K=4, graph="complete", lr=0.1, momentum=0.0, x0_shared=True)
+    out = _run_gpu(binding, inputs, w)
+    _compare(w, out)
+    want = out["x0"][0].astype(np.float64)
+    for g in out["grads"]:
+        want = want - w.lr * g.astype(np.float64).mean(axis=0)
+    assert_close("Z vs parallel SGD", out["Z"], np.broadcast_to(want, out["Z"].shape))
+
+
+def test_custom_four_node_graph_weights_converge(binding, inputs):
+    """The paper's worked 4-node matrix as a custom schedule: w -> (8,16,16,12)/13 and z -> average."""
+    rows = read_golden("four_node_update_equations.txt")
+    recv = [int(r[0]) for r in rows]; send = [int(r[1]) for r in rows]; wt = [float(eval(r[2])) for r in rows]
+    g = binding.GraphDesc.custom(1, [0] * len(rows), send, recv, wt)
+    from oracle import schedule as osched
+    P = osched.custom_mixing_matrix(4, send, recv, np.asarray(wt, dtype=np.float32))
+    w = inputs.Workload("four", n=4, d=300, K=60, graph="custom", lr=0.0, momentum=0.0, grad_std=0.0)
+    out = _run_gpu(binding, inputs, w, graph=g)
+    _compare(w, out, P_of_k=lambda k: P)
+    assert np.allclose(out["W"], np.array([8, 16, 16, 12]) / 13.0, rtol=1e-5)
+    assert np.allclose(out["Z"], np.broadcast_to(out["x0"].astype(np.float64).mean(axis=0), out["Z"].shape),
+                       rtol=0, atol=2e-6)
+
+
+def test_one_peer_consensus_on_gpu(binding, inputs):
+    """Zero gradients, n = 32: after log2(n) = 5 fused steps every node holds the average (fp32 rounding only)."""
+    w = inputs.Workload("consensus", n=32, d=1000, K=5, graph="exp", peers=1, lr=0.1, momentum=0.9, grad_std=0.0)
+    out = _run_gpu(binding, inputs, w)
+    mean = out["x0"].astype(np.float64).mean(axis=0)
+    assert np.abs(out["Z"] - mean).max() <= 4e-7 * np.abs(out["x0"]).max()
+
+
+def test_tile_and_grid_options_do_not_change_results(binding, inputs):
+    w = inputs.sweep_workload(16, 5000)
+    base = _run_gpu(binding, inputs, w)
+    for opts in ({"tile_cols": 32}, {"tile_cols": 1024}, {"ctas_per_sm": 1}, {"ctas_per_sm": 4}):
+        other = _run_gpu(binding, inputs, w, options=opts)
+        for name in ("X", "W", "M", "Z"):
+            assert np.array_equal(base[name], other[name], equal_nan=True), (opts, name)
+
+
+def test_standalone_debias(binding, inputs):
+    from oracle import sgp as osgp
+    for n, d, ld, off in ((5, 1027, 1027, 0), (16, 4096, 4100, 0), (3, 10, 12, 1)):
+        buf = torch.randn(n * ld + off + 4, device=DEV)
+        X = buf[off:off + n * ld].view(n, ld)[:, :d]
+        W = torch.rand(n, device=DEV) + 0.5
+        zb = torch.full((n * ld + off + 4,), float("nan"), device=DEV)
+        Z = zb[off:off + n * ld].view(n, ld)[:, :d]
+        with binding.Sgp(n, d, binding.GraphDesc.exp_peers(1), ld=ld) as h:
+            h.debias(X, W, Z)
+            torch.cuda.synchronize()
+        assert_close("Z", Z.cpu().numpy(), osgp.debias(X.cpu().numpy(), W.cpu().numpy()))
+        assert torch.isnan(zb).sum().item() == zb.numel() - n * d
+
+
+def test_ring_export_import_resumes_bit_exactly(binding, inputs):
+    import dataclasses
+    w = dataclasses.replace(inputs.sweep_workload(8, 1500), tau=2, K=9)
+    n, d = w.n, w.d
+    def fresh():
+        return (inputs.initial_x(w, device=DEV).contiguous(), torch.ones(n, device=DEV), torch.zeros((n, d), device=DEV),
+                torch.empty((n, d), device=DEV))
+    G = torch.empty((n, d), device=DEV)
+    X, W, M, Z = fresh()
+    with binding.Sgp(n, d, graph_desc(w, binding), tau=2) as h:
+        for k in range(9):
+            h.step(X, W, M, inputs.gradient(w, k, G), Z, k, w.lr, w.momentum, 0.0, True)
+        torch.cuda.synchronize()
+    X2, W2, M2, Z2 = fresh()
+    rx = torch.empty((2, n, d), device=DEV); rw = torch.empty((2, n), device=DEV)
+    with binding.Sgp(n, d, graph_desc(w, binding), tau=2) as h:
+        for k in range(4):
+            h.step(X2, W2, M2, inputs.gradient(w, k, G), Z2, k, w.lr, w.momentum, 0.0, True)
+        h.ring_export(rx, rw)
+        torch.cuda.synchronize()
+    with binding.Sgp(n, d, graph_desc(w, binding), tau=2) as h:
+        h.ring_import(rx, rw)
+        for k in range(4, 9):
+            h.step(X2, W2, M2, inputs.gradient(w, k, G), Z2, k, w.lr, w.momentum, 0.0, True)
+        torch.cuda.synchronize()
+    for a, b in ((X, X2), (W, W2), (M, M2), (Z, Z2)):
+        assert torch.equal(a, b)
+    with binding.Sgp(n, d, graph_desc(w, binding), tau=0) as h:
+        with pytest.raises(binding.SgpError) as ei:
+            h.ring_export(rx, rw)
+        assert ei.value.code == binding.SGP_ERR_STATE
+
+
+def test_step_host_matches_device_step(binding, inputs):
+    """Host-buffer entry point (chunked copy/compute pipeline) == device entry point, bit for bit."""
+    import dataclasses
+    for tau in (0, 1):
+        w = dataclasses.replace(inputs.sweep_workload(16, 50_004), tau=tau, K=4)
+        n, d = w.n, w.d
+        X = inputs.initial_x(w, device=DEV).contiguous(); W = torch.ones(n, device=DEV)
+        M = torch.zeros((n, d), device=DEV); Z = torch.empty((n, d), device=DEV); G = torch.empty((n, d), device=DEV)
+        X2, W2, M2 = X.clone(), W.clone(), M.clone()
+        dG = torch.empty((n, d), device=DEV); dZ = torch.empty((n, d), device=DEV)
+        hG = torch.empty((n, d), pin_memory=True); hZ = torch.empty((n, d), pin_memory=True)
+        with binding.Sgp(n, d, graph_desc(w, binding), tau=tau) as h1, binding.Sgp(n, d, graph_desc(w, binding), tau=tau) as h2:
+            for k in range(w.K):
+                inputs.gradient(w, k, G)
+                hG.copy_(G)
+                h1.step(X, W, M, G, Z, k, w.lr, w.momentum, 0.0, True)
+                torch.cuda.synchronize()
+                h2.step_host(X2, W2, M2, hG, hZ, dG, dZ, k, w.lr, w.momentum, 0.0, True, chunk_cols=8192)
+                assert torch.equal(hZ, Z.cpu())
+        assert torch.equal(X, X2) and torch.equal(W, W2) and torch.equal(M, M2)
+
+
+def test_invalid_step_arguments(binding, inputs):
+    n, d = 4, 64
+    X = torch.zeros((n, d), device=DEV); W = torch.ones(n, device=DEV); G = torch.zeros((n, d), device=DEV)
+    lib = binding.lib()
+    with binding.Sgp(n, d, binding.GraphDesc.exp_peers(1)) as h:
+        p = lambda t: t.data_ptr()
+        assert lib.sgp_step(h._h, p(X), p(W), None, p(G), None, -1, 0.1, 0.0, 0.0, 1, None) == binding.SGP_ERR_ARG
+        assert lib.sgp_step(h._h, p(X), p(W), None, p(G), None, 0, 0.1, 0.9, 0.0, 1, None) == binding.SGP_ERR_ARG
+        assert lib.sgp_step(h._h, None, p(W), None, p(G), None, 0, 0.1, 0.0, 0.0, 1, None) == binding.SGP_ERR_ARG
+        with pytest.raises(binding.SgpError):
+            h.set_option("no_such_knob", 1)
+        h.set_option("ctas_per_sm", 3)
+        assert h.get_option("ctas_per_sm") == 3

@@ -1,0 +1,164 @@
+"""Graph-schedule compiler (C++ host code behind the C ABI) against the oracle's generator: bit-exact
+in-neighbour lists and fp32 weights; validation of custom graphs; ABI surface.  CPU only."""
+import ctypes as C
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import schedule as S
+from conftest import ROOT, read_golden
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_1811_10792_b200 import build
+    build.build()
+    from paper_1811_10792_b200 import binding as b
+    return b
+
+
+def _assert_slot_equal(sched, k, P):
+    rowptr, col, val = sched.get(k)
+    o_rowptr, o_col, o_val = S.csr_in_neighbours(P)
+    assert np.array_equal(rowptr, o_rowptr)
+    assert np.array_equal(col, o_col)
+    want = o_val.astype(np.float32)
+    assert np.array_equal(val.view(np.int32), want.view(np.int32))      # bit-exact weights
+
+
+@pytest.mark.parametrize("n", [1, 2, 3, 4, 5, 8, 13, 16, 32, 64, 100, 256])
+@pytest.mark.parametrize("peers", [1, 2, 3])
+def test_exp_peers_bit_exact(binding, n, peers):
+    sched = binding.Schedule(n, binding.GraphDesc.exp_peers(peers))
+    assert sched.period == S.schedule_period("exp", n)
+    for k in range(2 * sched.period + 1):
+        _assert_slot_equal(sched, k, S.mixing_matrix("exp", n, k, peers=peers))
+
+
+@pytest.mark.parametrize("n", [1, 2, 7, 32, 256])
+def test_complete_bit_exact(binding, n):
+    sched = binding.Schedule(n, binding.GraphDesc.complete())
+    assert sched.period == 1
+    _assert_slot_equal(sched, 5, S.mixing_matrix("complete", n, 5))
+    assert sched.nnz(0) == n * n
+
+
+@pytest.mark.parametrize("n", [1, 2, 4, 16, 64, 256])
+@pytest.mark.parametrize("seed,max_outdeg,steps", [(181110797, 4, 10), (3, 1, 3), (2**63 + 5, 7, 4)])
+def test_random_outdeg_bit_exact(binding, n, seed, max_outdeg, steps):
+    sched = binding.Schedule(n, binding.GraphDesc.random_outdeg(seed, steps, max_outdeg))
+    assert sched.period == steps
+    for k in range(steps + 2):
+        _assert_slot_equal(sched, k, S.mixing_matrix("random", n, k, seed=seed, max_outdeg=max_outdeg,
+                                                     num_steps=steps))
+
+
+def _four_node_edges():
+    rows = read_golden("four_node_update_equations.txt")
+    recv = [int(r[0]) for r in rows]
+    send = [int(r[1]) for r in rows]
+    wt = [float(eval(r[2])) for r in rows]     # "1/2", "1/3"
+    return send, recv, wt
+
+
+def test_custom_graph_four_node_example(binding):
+    send, recv, wt = _four_node_edges()
+    g = binding.GraphDesc.custom(1, [0] * len(send), send, recv, wt)
+    sched = binding.Schedule(4, g)
+    P = S.custom_mixing_matrix(4, send, recv, np.asarray(wt, dtype=np.float32))
+    _assert_slot_equal(sched, 0, P)
+    rowptr, col, val = sched.get(0)
+    assert rowptr.tolist() == [0, 2, 5, 7, 9]
+    assert col.tolist() == [0, 3, 0, 1, 3, 1, 2, 2, 3]
+
+
+def test_custom_graph_two_steps_any_edge_order(binding):
+    # step 0: ring 0->1->2->0 with self-loops (1/2 each); step 1: node 0 broadcasts, others keep
+    step = [1, 0, 0, 0, 1, 0, 0, 1, 1, 0, 1]
+    send = [0, 2, 0, 1, 0, 0, 2, 2, 1, 1, 0]
+    recv = [2, 0, 1, 1, 1, 0, 2, 2, 1, 2, 0]
+    wt = [1 / 3, .5, .5, .5, 1 / 3, .5, .5, 1.0, 1.0, .5, 1 / 3]
+    sched = binding.Schedule(3, binding.GraphDesc.custom(2, step, send, recv, wt))
+    assert sched.period == 2
+    for k in (0, 1):
+        sel = [e for e in range(len(step)) if step[e] == k]
+        P = S.custom_mixing_matrix(3, [send[e] for e in sel], [recv[e] for e in sel],
+                                   np.asarray([wt[e] for e in sel], dtype=np.float32))
+        _assert_slot_equal(sched, k, P)
+        assert np.allclose(P.sum(axis=0), 1.0, atol=1e-7)
+
+
+@pytest.mark.parametrize("mutate", ["colsum", "no_self", "dup", "range", "neg", "nan", "step_range"])
+def test_custom_graph_rejected(binding, mutate):
+    send, recv, wt = _four_node_edges()
+    step = [0] * len(send)
+    if mutate == "colsum":
+        wt[0] = 0.6
+    elif mutate == "no_self":
+        # drop node 2's self-loop and give its whole mass to node 3
+        idx = [e for e in range(len(send)) if send[e] == 2 and recv[e] == 2][0]
+        del send[idx], recv[idx], wt[idx], step[idx]
+        wt[[e for e in range(len(send)) if send[e] == 2][0]] = 1.0
+    elif mutate == "dup":
+        send.append(send[0]); recv.append(recv[0]); wt.append(wt[0]); step.append(0)
+    elif mutate == "range":
+        recv[1] = 4
+    elif mutate == "neg":
+        wt[2] = -0.5
+    elif mutate == "nan":
+        wt[2] = float("nan")
+    elif mutate == "step_range":
+        step[3] = 1
+    with pytest.raises(binding.SgpError) as ei:
+        binding.Schedule(4, binding.GraphDesc.custom(1, step, send, recv, wt))
+    assert ei.value.code == binding.SGP_ERR_GRAPH
+
+
+def test_bad_arguments(binding):
+    for n in (0, -1, binding.SGP_MAX_NODES + 1):
+        with pytest.raises(binding.SgpError) as ei:
+            binding.Schedule(n, binding.GraphDesc.exp_peers(1))
+        assert ei.value.code == binding.SGP_ERR_ARG
+    for g in (binding.GraphDesc.exp_peers(0), binding.GraphDesc.random_outdeg(1, 0, 4),
+              binding.GraphDesc.random_outdeg(1, 5, 0), binding.GraphDesc(kind=17)):
+        with pytest.raises(binding.SgpError) as ei:
+            binding.Schedule(4, g)
+        assert ei.value.code == binding.SGP_ERR_ARG
+    sched = binding.Schedule(4, binding.GraphDesc.exp_peers(1))
+    lib = binding.lib()
+    nnz = C.c_int64()
+    small = np.zeros(2, dtype=np.int32)
+    rowptr = np.zeros(5, dtype=np.int32)
+    assert lib.sgp_schedule_get(sched._ptr, 0, rowptr.ctypes.data, small.ctypes.data, small.ctypes.data, 2,
+                                C.byref(nnz)) == binding.SGP_ERR_ARG
+    assert nnz.value == 8
+    assert lib.sgp_schedule_get(sched._ptr, -1, rowptr.ctypes.data, small.ctypes.data, small.ctypes.data, 2,
+                                C.byref(nnz)) == binding.SGP_ERR_ARG
+    assert lib.sgp_schedule_period(None, C.byref(nnz)) == binding.SGP_ERR_ARG
+    assert binding.strerror(binding.SGP_ERR_GRAPH).startswith("schedule")
+
+
+def test_library_exports_every_declared_symbol(binding):
+    header = open(os.path.join(ROOT, "include", "sgp.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(sgp_[a-z_0-9]+)\s*\(", header))
+    assert declared == set(binding.EXPORTS), declared ^ set(binding.EXPORTS)
+    lib = binding.lib()
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert binding.version() >= 100
+
+
+def test_handle_calls_reject_null_without_a_gpu(binding):
+    lib = binding.lib()
+    assert lib.sgp_step(None, None, None, None, None, None, 0, 0.1, 0.0, 0.0, 1, None) == binding.SGP_ERR_ARG
+    assert lib.sgp_debias(None, None, None, None, None) == binding.SGP_ERR_ARG
+    assert lib.sgp_destroy(None) == binding.SGP_OK
+    out = C.c_void_p()
+    g = binding.GraphDesc.exp_peers(1)
+    assert lib.sgp_create(C.byref(out), 0, 10, 10, C.byref(g.c), 0, 0) == binding.SGP_ERR_ARG
+    assert lib.sgp_create(C.byref(out), 4, 10, 8, C.byref(g.c), 0, 0) == binding.SGP_ERR_ARG      # ld < d
+    assert lib.sgp_create(C.byref(out), 4, 10, 10, C.byref(g.c), -1, 0) == binding.SGP_ERR_ARG    # tau < 0
+    assert out.value is None
