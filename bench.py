@@ -188,6 +188,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--option", action="append", default=[], help="key=value passed to sgp_set_option")
+    ap.add_argument("--ld-align", type=int, default=256,
+                    help="row pitch of every n x d array is rounded up to this many floats (256 = 1 KB rows)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -220,16 +222,23 @@ def main():
     arr_bytes = 4 * n * d
     n_state = 3 + (1 if w.tau else 0)                       # X, M, Z (+ ring inside the handle)
     pool = max(1, min(K, int((free_b * 0.6 - n_state * arr_bytes) // arr_bytes)))
-    X = inputs.initial_x(w, device=dev).contiguous()
-    M = torch.zeros_like(X) if w.momentum != 0.0 else None
-    Z = torch.empty_like(X)
+    ld = (d + args.ld_align - 1) // args.ld_align * args.ld_align
+
+    def matrix():
+        # n x d view of an n x ld allocation: rows start on 1 KB boundaries when ld is a multiple of 256
+        return torch.zeros((n, ld), dtype=torch.float32, device=dev)[:, :d]
+
+    X = matrix()
+    X.copy_(inputs.initial_x(w, device=dev))
+    M = matrix() if w.momentum != 0.0 else None
+    Z = matrix()
     Wt = torch.ones(n, device=dev)
     Gs = []
     for k in range(pool):
-        G = torch.empty_like(X)
+        G = matrix()
         inputs.gradient(w, k, G)
         Gs.append(G)
-    h = binding.Sgp(n, d, graph_desc(w, binding), tau=w.tau)
+    h = binding.Sgp(n, d, graph_desc(w, binding), tau=w.tau, ld=ld)
     for kv in args.option:
         key, val = kv.split("=")
         h.set_option(key, int(val))
@@ -267,8 +276,8 @@ def main():
     # ---- end to end through the host-buffer entry point (gradients in, de-biased parameters out)
     e2e = None
     if not args.no_e2e:
-        hG = torch.empty((n, d), dtype=torch.float32, pin_memory=True)
-        hZ = torch.empty((n, d), dtype=torch.float32, pin_memory=True)
+        hG = torch.empty((n, ld), dtype=torch.float32, pin_memory=True)[:, :d]
+        hZ = torch.empty((n, ld), dtype=torch.float32, pin_memory=True)[:, :d]
         hG.copy_(Gs[0])
         dG = Gs[0]
         torch.cuda.synchronize()
@@ -311,7 +320,8 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
             "ms_per_step": max_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
-            "config": workload_config(w, extra={"gradient_pool": pool, "parallelism": f"replicas x{world}"}),
+            "config": workload_config(w, extra={"gradient_pool": pool, "parallelism": f"replicas x{world}",
+                                                "row_pitch_floats": ld}),
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": K, "clocks": sampler.summary(),
         }
         print(json.dumps(line), flush=True)

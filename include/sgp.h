@@ -162,9 +162,11 @@ int sgp_check(sgp_handle *h, const float *d_X, const float *d_W, double *h_stats
 
 /*
  * Tuning knobs for experiments (defaults are chosen per problem shape):
- *   "variant"      0 = automatic, 1 = register-staged kernel, 2 = bulk-copy (TMA) pipelined kernel
+ *   "variant"      0 = automatic, 1 = register-staged kernel, 2 = TMA pipelined kernel fed by 2-D tensor
+ *                  maps, 3 = the same kernel fed by one bulk copy per row segment (no tensor maps)
  *   "tile_cols"    columns per tile (multiple of 4; 0 = automatic)
  *   "ctas_per_sm"  persistent CTAs per SM (0 = automatic)
+ *   "stages"       shared-memory stages of the bulk-copy pipeline (0 = automatic, at most 8)
  * Unknown keys or unsupported values return SGP_ERR_ARG and change nothing.
  */
 int sgp_set_option(sgp_handle *h, const char *key, int64_t value);

@@ -35,10 +35,19 @@ struct sgp_handle {
   float *ring_w = nullptr;   // tau * n
   unsigned *d_words = nullptr;  // [0] ticket, [1] status
   double *d_stats = nullptr;    // 4 doubles for sgp_check
-  int64_t opt_variant = 0, opt_tile_cols = 0, opt_ctas_per_sm = 0;
+  int64_t opt_variant = 0, opt_tile_cols = 0, opt_ctas_per_sm = 0, opt_stages = 0;
   cudaStream_t s_h2d = nullptr, s_compute = nullptr, s_d2h = nullptr;
   std::vector<cudaEvent_t> ev_in, ev_done;
   int last_cuda_error = 0;
+  // tensor maps already encoded for (base pointer, box columns)
+  struct MapEntry {
+    const void *ptr;
+    int box_cols;
+    CUtensorMap map;
+  };
+  std::vector<MapEntry> map_cache;
+  void *encode_fn = nullptr;   // cuTensorMapEncodeTiled, resolved lazily through the runtime
+  bool encode_tried = false;
 };
 
 namespace {
@@ -96,6 +105,20 @@ StepKernel pick_update(bool has_m, bool nesterov, bool has_z, bool has_ring) {
   return nesterov ? pick_z<VEC, true, true>(has_z, has_ring) : pick_z<VEC, true, false>(has_z, has_ring);
 }
 
+using TmaKernel = void (*)(const StepParams, const ConstTable, const sgp::TmaMaps, const int, const int);
+
+template <bool HAS_M, bool NESTEROV>
+TmaKernel pick_tma_z(bool has_z, bool has_ring) {
+  if (has_z) return has_ring ? sgp::sgp_step_tma_kernel<HAS_M, NESTEROV, true, true>
+                             : sgp::sgp_step_tma_kernel<HAS_M, NESTEROV, true, false>;
+  return has_ring ? sgp::sgp_step_tma_kernel<HAS_M, NESTEROV, false, true>
+                  : sgp::sgp_step_tma_kernel<HAS_M, NESTEROV, false, false>;
+}
+TmaKernel pick_tma(bool has_m, bool nesterov, bool has_z, bool has_ring) {
+  if (!has_m) return pick_tma_z<false, false>(has_z, has_ring);
+  return nesterov ? pick_tma_z<true, true>(has_z, has_ring) : pick_tma_z<true, false>(has_z, has_ring);
+}
+
 struct StepArgs {
   float *X, *W, *M;
   const float *G;
@@ -105,8 +128,8 @@ struct StepArgs {
   int nesterov;
 };
 
-// One launch of the register-staged kernel over columns [c0, c1) with vector width vec.
-int launch_regs(sgp_handle *h, const StepArgs &a, int64_t c0, int64_t c1, int vec, bool update_w, cudaStream_t stream) {
+// Fills the launch-independent part of the kernel arguments for step a.k.
+void fill_params(const sgp_handle *h, const StepArgs &a, int64_t c0, int64_t c1, bool update_w, StepParams *out) {
   const int64_t slot = a.k % h->sched->period();
   const SgpStepCsr &csr = h->sched->slot(a.k);
   StepParams p{};
@@ -134,14 +157,65 @@ int launch_regs(sgp_handle *h, const StepArgs &a, int64_t c0, int64_t c1, int ve
   p.val = h->d_val + h->off_nnz[static_cast<size_t>(slot)];
   p.ticket = h->d_words;
   p.status = h->d_words + 1;
+  *out = p;
+}
+
+// Launch plan of one step: which kernel, how wide a tile, how deep a pipeline, how many CTAs per SM.
+struct Plan {
+  int variant;        // 1 register-staged, 2 TMA with tensor maps, 3 TMA with per-row bulk copies
+  int64_t tile_cols;  // 0 = kernel default
+  int stages;
+  int cps;
+};
+
+size_t table_smem_bytes(const sgp_handle *h, int nnz) { return (static_cast<size_t>(h->n) + 1 + 2 * static_cast<size_t>(nnz)) * 4; }
+
+// Heuristics from measurements on B200.  The step is HBM-bound; what decides the achieved bandwidth
+// is the length of the contiguous row segments (>= 1 KB), the bytes in flight per SM and a grid that
+// is exactly one wave.  Measured (fraction of the copy bandwidth, rows on 1 KB boundaries):
+//   momentum, n <= 16 : register-staged 0.97, TMA 0.90      momentum, n = 32 : TMA 0.97, register-staged 0.95
+//   no momentum, n=16 : TMA 0.96, register-staged 0.87      tau = 1, n = 32  : register-staged 0.97
+// cps = 0 means "as many CTAs per SM as are resident" (asked of the occupancy calculator at launch).
+// Explicit options override each field.
+Plan make_plan(const sgp_handle *h, int arrays, bool has_m, int nnz, bool vec) {
+  Plan pl{1, 0, 2, 0};
+  if (vec) {
+    const size_t fixed = 16 * sizeof(uint64_t) + 3 * static_cast<size_t>(h->n) * 4 + 1024 +
+                         (table_smem_bytes(h, nnz) <= 40 * 1024 ? table_smem_bytes(h, nnz) : 0);
+    const size_t per_kb = static_cast<size_t>(arrays) * h->n * 1024;   // one stage at 1 KB per row segment
+    const size_t half_sm = 112 * 1024, full_sm = 224 * 1024;
+    if (!has_m && 2 * per_kb + fixed <= half_sm) {
+      pl = Plan{3, 256, 2, 2};
+    } else if (has_m && h->n > 16 && 2 * per_kb + fixed <= full_sm) {
+      pl = Plan{3, 256, 2, 2 * per_kb + fixed <= half_sm ? 2 : 1};
+    } else {
+      // register-staged: 1 KB row segments, or about 1024 vector items per tile when n is small;
+      // the double-buffered exchange tile is 2 x n x tile_cols x 4 bytes
+      pl.tile_cols = std::max<int64_t>(256, int64_t{4} << floor_log2(std::max<int64_t>(1, 1024 / h->n)));
+      while (pl.tile_cols > 32 && 2 * static_cast<size_t>(h->n) * pl.tile_cols * 4 + fixed > 100 * 1024) pl.tile_cols >>= 1;
+    }
+  }
+  if (h->opt_variant > 0) pl.variant = static_cast<int>(h->opt_variant);
+  if (h->opt_tile_cols > 0) pl.tile_cols = h->opt_tile_cols;
+  if (h->opt_stages > 0) pl.stages = static_cast<int>(h->opt_stages);
+  if (h->opt_ctas_per_sm > 0) pl.cps = static_cast<int>(h->opt_ctas_per_sm);
+  return pl;
+}
+
+// One launch of the register-staged kernel over columns [c0, c1) with vector width vec.
+int launch_regs(sgp_handle *h, const StepArgs &a, const Plan &pl, int64_t c0, int64_t c1, int vec, bool update_w,
+                cudaStream_t stream) {
+  const int64_t slot = a.k % h->sched->period();
+  StepParams p{};
+  fill_params(h, a, c0, c1, update_w, &p);
 
   // tile width: about kThreads * kItemsPerThread items per tile, at least 128 bytes per row segment
   const int64_t ncols = c1 - c0;
   const int min_tv = vec == 4 ? 8 : 32;
   int64_t tv = int64_t{1} << floor_log2(std::max<int64_t>(1, sgp::kThreads * sgp::kItemsPerThread / h->n));
-  if (h->opt_tile_cols > 0) tv = int64_t{1} << floor_log2(std::max<int64_t>(1, h->opt_tile_cols / vec));
+  if (pl.tile_cols > 0) tv = int64_t{1} << floor_log2(std::max<int64_t>(1, pl.tile_cols / vec));
   tv = std::max<int64_t>(tv, min_tv);
-  const size_t table_bytes = (static_cast<size_t>(h->n) + 1 + 2 * static_cast<size_t>(p.nnz)) * 4;
+  const size_t table_bytes = table_smem_bytes(h, p.nnz);
   if (h->const_ok[static_cast<size_t>(slot)]) p.table_mode = 0;
   else p.table_mode = table_bytes <= 40 * 1024 ? 1 : 2;
   size_t smem = 0;
@@ -155,18 +229,111 @@ int launch_regs(sgp_handle *h, const StepArgs &a, int64_t c0, int64_t c1, int ve
   p.log2_tile_vecs = floor_log2(tv);
   const int64_t tile_cols = tv * vec;
   const int64_t ntiles = (ncols + tile_cols - 1) / tile_cols;
-  const int cps = h->opt_ctas_per_sm > 0 ? static_cast<int>(h->opt_ctas_per_sm) : 2;
-  const int64_t grid = std::min<int64_t>(ntiles, static_cast<int64_t>(h->sm_count) * cps);
-
   const bool has_m = a.momentum != 0.0f;
   StepKernel kern = vec == 4 ? pick_update<4>(has_m, a.nesterov != 0, a.Z != nullptr, h->tau > 0)
                              : pick_update<1>(has_m, a.nesterov != 0, a.Z != nullptr, h->tau > 0);
   if (smem > 48 * 1024)
     SGP_CUDA_TRY(h, cudaFuncSetAttribute(reinterpret_cast<const void *>(kern),
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  int cps = pl.cps;
+  if (cps <= 0) {   // persistent grid of exactly one wave
+    SGP_CUDA_TRY(h, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&cps, reinterpret_cast<const void *>(kern),
+                                                                  sgp::kThreads, smem));
+    cps = std::max(1, cps);
+  }
+  const int64_t grid = std::min<int64_t>(ntiles, static_cast<int64_t>(h->sm_count) * cps);
   static const ConstTable kEmptyTable{};
   const ConstTable &ct = p.table_mode == 0 ? h->const_tables[static_cast<size_t>(slot)] : kEmptyTable;
   kern<<<static_cast<unsigned>(grid), sgp::kThreads, smem, stream>>>(p, ct);
+  SGP_CUDA_TRY(h, cudaGetLastError());
+  return SGP_OK;
+}
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// Tensor map of an n x d fp32 array with row pitch ld whose box is (box_cols x n); cached per pointer.
+// Returns false when the driver entry point is unavailable or the encoding is rejected.
+bool get_tensor_map(sgp_handle *h, const float *base, int box_cols, CUtensorMap *out) {
+  for (const auto &e : h->map_cache)
+    if (e.ptr == base && e.box_cols == box_cols) {
+      *out = e.map;
+      return true;
+    }
+  if (!h->encode_tried) {
+    h->encode_tried = true;
+    cudaDriverEntryPointQueryResult qres;
+    void *fn = nullptr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      h->encode_fn = fn;
+    else
+      (void)cudaGetLastError();
+  }
+  if (h->encode_fn == nullptr || h->d >= (int64_t{1} << 31)) return false;
+  const cuuint64_t gdim[2] = {static_cast<cuuint64_t>(h->d), static_cast<cuuint64_t>(h->n)};
+  const cuuint64_t gstride[1] = {static_cast<cuuint64_t>(h->ld) * sizeof(float)};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(box_cols), static_cast<cuuint32_t>(h->n)};
+  const cuuint32_t estride[2] = {1, 1};
+  CUtensorMap m;
+  const CUresult r = reinterpret_cast<EncodeTiledFn>(h->encode_fn)(
+      &m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float *>(base), gdim, gstride, box, estride,
+      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return false;
+  if (h->map_cache.size() >= 256) h->map_cache.clear();
+  h->map_cache.push_back({base, box_cols, m});
+  *out = m;
+  return true;
+}
+
+// One launch of the bulk-copy pipelined kernel over columns [c0, c1) (needs the 128-bit preconditions).
+// Returns SGP_ERR_STATE when the shape does not fit its shared-memory stages; the caller then uses
+// the register-staged kernel.
+int launch_tma(sgp_handle *h, const StepArgs &a, const Plan &pl, int64_t c0, int64_t c1, bool update_w,
+               cudaStream_t stream) {
+  const int64_t slot = a.k % h->sched->period();
+  StepParams p{};
+  fill_params(h, a, c0, c1, update_w, &p);
+  const bool has_m = a.momentum != 0.0f, has_ring = h->tau > 0;
+  const int arrays = 2 + (has_m ? 1 : 0) + (has_ring ? 1 : 0);
+  int64_t tv = int64_t{1} << floor_log2(std::max<int64_t>(1, (pl.tile_cols > 0 ? pl.tile_cols : 256) / 4));
+  tv = std::max<int64_t>(tv, 8);
+  int stages = std::max(1, pl.stages);
+  const int cps = pl.cps > 0 ? pl.cps : 2;
+  const size_t table_bytes = table_smem_bytes(h, p.nnz);
+  if (h->const_ok[static_cast<size_t>(slot)]) p.table_mode = 0;
+  else p.table_mode = table_bytes <= 40 * 1024 ? 1 : 2;
+  const size_t fixed = 16 * sizeof(uint64_t) + 3 * static_cast<size_t>(h->n) * 4 + (p.table_mode < 2 ? table_bytes : 0);
+  const size_t budget = std::min<size_t>(static_cast<size_t>(h->smem_optin), (228 * 1024) / static_cast<size_t>(cps) - 2048);
+  size_t smem = 0;
+  for (;;) {
+    smem = static_cast<size_t>(stages) * arrays * h->n * tv * 16 + fixed;
+    if (smem <= budget) break;
+    if (h->opt_stages == 0 && stages > 2) --stages;
+    else if (h->opt_tile_cols == 0 && tv > 8) tv >>= 1;
+    else return SGP_ERR_STATE;
+  }
+  p.log2_tile_vecs = floor_log2(tv);
+  const int64_t tile_cols = tv * 4;
+  const int64_t ntiles = (c1 - c0 + tile_cols - 1) / tile_cols;
+  const int64_t grid = std::min<int64_t>(ntiles, static_cast<int64_t>(h->sm_count) * cps);
+  TmaKernel kern = pick_tma(has_m, a.nesterov != 0, a.Z != nullptr, has_ring);
+  if (smem > 48 * 1024)
+    SGP_CUDA_TRY(h, cudaFuncSetAttribute(reinterpret_cast<const void *>(kern),
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  static const ConstTable kEmptyTable{};
+  const ConstTable &ct = p.table_mode == 0 ? h->const_tables[static_cast<size_t>(slot)] : kEmptyTable;
+  // 2-D tensor maps (one copy per array per tile) when the box fits; else one bulk copy per row segment
+  sgp::TmaMaps maps;
+  std::memset(&maps, 0, sizeof(maps));
+  bool use_maps = pl.variant == 2 && tile_cols <= 256 && tile_cols * 4 % 128 == 0;
+  if (use_maps) use_maps = get_tensor_map(h, a.X, static_cast<int>(tile_cols), &maps.x);
+  if (use_maps) use_maps = get_tensor_map(h, a.G, static_cast<int>(tile_cols), &maps.g);
+  if (use_maps && has_m) use_maps = get_tensor_map(h, a.M, static_cast<int>(tile_cols), &maps.m);
+  if (use_maps && has_ring) use_maps = get_tensor_map(h, p.ring_x, static_cast<int>(tile_cols), &maps.r);
+  kern<<<static_cast<unsigned>(grid), sgp::kTmaThreads, smem, stream>>>(p, ct, maps, stages, use_maps ? 1 : 0);
   SGP_CUDA_TRY(h, cudaGetLastError());
   return SGP_OK;
 }
@@ -176,11 +343,20 @@ int launch_step_range(sgp_handle *h, const StepArgs &a, int64_t c0, int64_t c1, 
   const bool vec_ok = aligned16(a.X) && aligned16(a.G) && (a.M == nullptr || aligned16(a.M)) &&
                       (a.Z == nullptr || aligned16(a.Z)) && (h->ld % 4 == 0) && (c0 % 4 == 0);
   const int64_t vec_end = vec_ok ? c0 + ((c1 - c0) & ~int64_t{3}) : c0;
+  const int arrays = 2 + (a.M != nullptr ? 1 : 0) + (h->tau > 0 ? 1 : 0);
+  const int nnz = static_cast<int>(h->sched->slot(a.k).col.size());
   if (vec_end > c0) {
-    const int rc = launch_regs(h, a, c0, vec_end, 4, update_w && vec_end == c1, stream);
+    const Plan pl = make_plan(h, arrays, a.M != nullptr, nnz, true);
+    int rc = SGP_ERR_STATE;
+    if (pl.variant >= 2) rc = launch_tma(h, a, pl, c0, vec_end, update_w && vec_end == c1, stream);
+    if (rc == SGP_ERR_STATE) {
+      Plan fallback = pl;
+      if (pl.variant >= 2 && h->opt_ctas_per_sm == 0) fallback.cps = 0;
+      rc = launch_regs(h, a, fallback, c0, vec_end, 4, update_w && vec_end == c1, stream);
+    }
     if (rc != SGP_OK) return rc;
   }
-  if (vec_end < c1) return launch_regs(h, a, vec_end, c1, 1, update_w, stream);
+  if (vec_end < c1) return launch_regs(h, a, make_plan(h, arrays, a.M != nullptr, nnz, false), vec_end, c1, 1, update_w, stream);
   return SGP_OK;
 }
 
@@ -438,7 +614,7 @@ int sgp_check(sgp_handle *h, const float *d_X, const float *d_W, double *h_stats
 int sgp_set_option(sgp_handle *h, const char *key, int64_t value) {
   if (h == nullptr || key == nullptr || value < 0) return SGP_ERR_ARG;
   if (std::strcmp(key, "variant") == 0) {
-    if (value > 2) return SGP_ERR_ARG;
+    if (value > 3) return SGP_ERR_ARG;
     h->opt_variant = value;
   } else if (std::strcmp(key, "tile_cols") == 0) {
     if (value % 4 != 0 || value > 4096) return SGP_ERR_ARG;
@@ -446,6 +622,9 @@ int sgp_set_option(sgp_handle *h, const char *key, int64_t value) {
   } else if (std::strcmp(key, "ctas_per_sm") == 0) {
     if (value > 16) return SGP_ERR_ARG;
     h->opt_ctas_per_sm = value;
+  } else if (std::strcmp(key, "stages") == 0) {
+    if (value > 8) return SGP_ERR_ARG;
+    h->opt_stages = value;
   } else {
     return SGP_ERR_ARG;
   }
@@ -457,6 +636,7 @@ int sgp_get_option(const sgp_handle *h, const char *key, int64_t *value) {
   if (std::strcmp(key, "variant") == 0) *value = h->opt_variant;
   else if (std::strcmp(key, "tile_cols") == 0) *value = h->opt_tile_cols;
   else if (std::strcmp(key, "ctas_per_sm") == 0) *value = h->opt_ctas_per_sm;
+  else if (std::strcmp(key, "stages") == 0) *value = h->opt_stages;
   else return SGP_ERR_ARG;
   return SGP_OK;
 }

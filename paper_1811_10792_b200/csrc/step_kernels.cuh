@@ -6,6 +6,7 @@
 // delayed-message ring (Alg. 2), de-bias (Alg. 1 line 8) -- with one read and one write of each
 // array and no inter-CTA dependency (no grid sync, no device-side wait on another CTA).
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -167,7 +168,7 @@ template <int VEC, bool HAS_M, bool NESTEROV, bool HAS_Z, bool HAS_RING>
 __global__ void __launch_bounds__(kThreads, 2)
 sgp_step_regs_kernel(const __grid_constant__ StepParams p, const __grid_constant__ ConstTable ct) {
   using V = typename VecT<VEC>::type;
-  extern __shared__ __align__(16) unsigned char smem_raw[];
+  extern __shared__ __align__(128) unsigned char smem_raw[];
   const int n = p.n;
   const int tv = 1 << p.log2_tile_vecs;
   const int tile_items = n * tv;
@@ -262,6 +263,248 @@ sgp_step_regs_kernel(const __grid_constant__ StepParams p, const __grid_constant
       }
     }
     buf ^= 1;
+  }
+}
+
+}  // namespace sgp
+
+namespace sgp {
+
+// ------------------------------------------------------------------------------------------------
+// Bulk-copy (TMA) pipelined kernel.  A producer warp streams whole column tiles -- every node's row
+// segment of X, G (and M, ring) -- into a ring of shared-memory stages with cp.async.bulk, completion
+// counted on an mbarrier per stage; eight consumer warps update, exchange through the stage itself
+// (x^(k+1/2) overwrites the X tile in place), gather-mix and store with 128-bit streaming stores.
+// Loads therefore stay in flight while the consumers compute and store.  No multicast, no cluster.
+// Every wait is bounded: on expiry the CTA records a status bit and leaves.
+// ------------------------------------------------------------------------------------------------
+constexpr int kTmaConsumers = 256;
+constexpr int kTmaThreads = kTmaConsumers + 32;
+constexpr unsigned kStatusFullTimeout = 1u;
+constexpr unsigned kStatusEmptyTimeout = 2u;
+constexpr unsigned kStatusDrainTimeout = 4u;
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Waits for the phase with the given parity; gives up after about two seconds.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_timer_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (global_timer_ns() - t0 > 2000000000ull) return false;
+  }
+}
+// One contiguous global -> shared copy of `bytes` (multiple of 16, both addresses 16-byte aligned).
+__device__ __forceinline__ void bulk_copy_g2s(void *dst_smem, const void *src_gmem, uint32_t bytes, uint64_t *bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(dst_smem)),
+               "l"(__cvta_generic_to_global(src_gmem)), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+// Tiled 2-D tensor copy global -> shared: box of (tile columns x all n rows) at column x, row y.
+__device__ __forceinline__ void tma_load_2d(void *dst_smem, const CUtensorMap *map, int x, int y, uint64_t *bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+          smem_u32(dst_smem)),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar))
+      : "memory");
+}
+// Tensor maps of the arrays a launch streams in (only those the launch uses are encoded).
+struct alignas(64) TmaMaps {
+  CUtensorMap x, g, m, r;
+};
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void consumer_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kTmaConsumers) : "memory"); }
+// Barrier over the consumer threads that also ANDs a flag, so that all of them take the same decision.
+__device__ __forceinline__ bool consumer_all(bool flag) {
+  uint32_t out;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %1, 0;\n\t"
+      "bar.red.and.pred p, 1, %2, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(out)
+      : "r"(static_cast<uint32_t>(flag)), "n"(kTmaConsumers)
+      : "memory");
+  return out != 0;
+}
+
+template <bool HAS_M, bool NESTEROV, bool HAS_Z, bool HAS_RING>
+__global__ void __launch_bounds__(kTmaThreads, 2)
+sgp_step_tma_kernel(const __grid_constant__ StepParams p, const __grid_constant__ ConstTable ct,
+                    const __grid_constant__ TmaMaps maps, const int stages, const int use_tensor_maps) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  constexpr int kArrays = 2 + (HAS_M ? 1 : 0) + (HAS_RING ? 1 : 0);
+  constexpr int kMaxStages = 8;
+  const int n = p.n;
+  const int tv = 1 << p.log2_tile_vecs;
+  const int tile_items = n * tv;                       // float4 items per array per stage
+  const size_t stage_bytes = static_cast<size_t>(kArrays) * tile_items * sizeof(float4);
+  uint64_t *full_bar = reinterpret_cast<uint64_t *>(smem_raw + stages * stage_bytes);
+  uint64_t *empty_bar = full_bar + kMaxStages;
+  float *scratch = reinterpret_cast<float *>(empty_bar + kMaxStages);
+  __shared__ int s_abort;
+
+  const CtaTables tab = cta_prologue<HAS_RING>(p, ct, scratch, kTmaThreads);
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(full_bar + s, 1);
+      mbar_init(empty_bar + s, kTmaConsumers / 32);
+    }
+    s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  const int64_t ld = p.ld;
+  const int64_t ncols = p.col_end - p.col_begin;
+  const int64_t tile_cols = static_cast<int64_t>(tv) * 4;
+  const int64_t ntiles = (ncols + tile_cols - 1) / tile_cols;
+  const int64_t my_tiles = ntiles > blockIdx.x ? (ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  volatile int *abort_flag = &s_abort;
+
+  if (warp == kTmaConsumers / 32) {
+    // ---------------- producer warp
+    int64_t issued = 0;
+    for (int64_t it = 0; it < my_tiles && !*abort_flag; ++it) {
+      const int s = static_cast<int>(it % stages);
+      const int64_t round = it / stages;
+      if (round > 0 && !mbar_wait_bounded(empty_bar + s, static_cast<uint32_t>((round - 1) & 1))) {
+        if (lane == 0) atomicOr(p.status, kStatusEmptyTimeout);
+        *abort_flag = 1;
+        break;
+      }
+      const int64_t tile = blockIdx.x + it * gridDim.x;
+      const int64_t col0 = p.col_begin + tile * tile_cols;
+      const int64_t valid = min(tile_cols, p.col_end - col0);
+      const uint32_t seg_bytes = static_cast<uint32_t>(valid * 4);
+      unsigned char *stage = smem_raw + s * stage_bytes;
+      if (use_tensor_maps) {
+        // one box per array: tile columns x n rows; columns past d are zero-filled by the copy engine
+        if (lane == 0) {
+          const size_t arr_bytes = static_cast<size_t>(tile_items) * sizeof(float4);
+          mbar_arrive_expect_tx(full_bar + s, static_cast<uint32_t>(stage_bytes));
+          tma_load_2d(stage, &maps.x, static_cast<int>(col0), 0, full_bar + s);
+          tma_load_2d(stage + arr_bytes, &maps.g, static_cast<int>(col0), 0, full_bar + s);
+          if (HAS_M) tma_load_2d(stage + 2 * arr_bytes, &maps.m, static_cast<int>(col0), 0, full_bar + s);
+          if (HAS_RING)
+            tma_load_2d(stage + (2 + (HAS_M ? 1 : 0)) * arr_bytes, &maps.r, static_cast<int>(col0), 0, full_bar + s);
+        }
+        issued = it + 1;
+        continue;
+      }
+      if (lane == 0) mbar_arrive_expect_tx(full_bar + s, seg_bytes * static_cast<uint32_t>(n * kArrays));
+      __syncwarp();
+      for (int c = lane; c < n * kArrays; c += 32) {
+        const int arr = c / n, row = c - arr * n;
+        const float *src;
+        if (arr == 0) src = p.X;
+        else if (arr == 1) src = p.G;
+        else if (arr == 2 && HAS_M) src = p.M;
+        else src = p.ring_x;
+        bulk_copy_g2s(stage + (static_cast<size_t>(arr) * tile_items + static_cast<size_t>(row) * tv) * sizeof(float4),
+                      src + static_cast<int64_t>(row) * ld + col0, seg_bytes, full_bar + s);
+      }
+      issued = it + 1;
+    }
+    // On an aborted run copies may still be in flight to this CTA's shared memory: wait for them (bounded).
+    if (*abort_flag) {
+      for (int64_t it = (issued > stages ? issued - stages : 0); it < issued; ++it) {
+        const int s = static_cast<int>(it % stages);
+        if (!mbar_wait_bounded(full_bar + s, static_cast<uint32_t>((it / stages) & 1)) && lane == 0)
+          atomicOr(p.status, kStatusDrainTimeout);
+      }
+    }
+  } else {
+    // ---------------- consumer warps
+    const float lr = p.lr, momentum = p.momentum, wd = p.wd;
+    const int ctid = threadIdx.x;
+    for (int64_t it = 0; it < my_tiles; ++it) {
+      const int s = static_cast<int>(it % stages);
+      const int64_t round = it / stages;
+      // bounded wait, then a vote: either every consumer goes on or every consumer leaves
+      const bool arrived = !*abort_flag && mbar_wait_bounded(full_bar + s, static_cast<uint32_t>(round & 1));
+      if (!consumer_all(arrived)) {
+        if (ctid == 0) atomicOr(p.status, kStatusFullTimeout);
+        *abort_flag = 1;
+        break;
+      }
+      const int64_t tile = blockIdx.x + it * gridDim.x;
+      const int64_t col0 = p.col_begin + tile * tile_cols;
+      float4 *Xs = reinterpret_cast<float4 *>(smem_raw + s * stage_bytes);
+      const float4 *Gs = Xs + tile_items;
+      const float4 *Ms = Gs + tile_items;
+      const float4 *Rs = Xs + static_cast<size_t>(2 + (HAS_M ? 1 : 0)) * tile_items;
+      // phase 1: local update; x^(k+1/2) replaces x in the stage
+      for (int item = ctid; item < tile_items; item += kTmaConsumers) {
+        const int row = item >> p.log2_tile_vecs;
+        const int c = item & (tv - 1);
+        const int64_t col = col0 + static_cast<int64_t>(c) * 4;
+        if (col < p.col_end) {
+          float4 u = HAS_M ? Ms[item] : make_float4(0.f, 0.f, 0.f, 0.f);
+          const float4 h = local_update<HAS_M, NESTEROV, float4>(Xs[item], Gs[item], u, lr, momentum, wd);
+          if (HAS_M) st_stream(reinterpret_cast<float4 *>(p.M + static_cast<int64_t>(row) * ld + col), u);
+          Xs[item] = h;
+        }
+      }
+      consumer_barrier();
+      // phase 2: gather-mix, ring exchange, de-bias
+      for (int item = ctid; item < tile_items; item += kTmaConsumers) {
+        const int row = item >> p.log2_tile_vecs;
+        const int c = item & (tv - 1);
+        const int64_t col = col0 + static_cast<int64_t>(c) * 4;
+        if (col < p.col_end) {
+          const int64_t o = static_cast<int64_t>(row) * ld + col;
+          float4 acc = make_float4(0.f, 0.f, 0.f, 0.f), offd = acc;
+          const int e1 = tab.rowptr[row + 1];
+          for (int e = tab.rowptr[row]; e < e1; ++e) {
+            const int j = tab.col[e];
+            const float pv = tab.val[e];
+            const float4 hj = Xs[(j << p.log2_tile_vecs) + c];
+            if (HAS_RING && j != row) offd = vfma(pv, hj, offd);
+            else acc = vfma(pv, hj, acc);
+          }
+          if (HAS_RING) {
+            acc = vadd(acc, Rs[item]);
+            st_stream(reinterpret_cast<float4 *>(p.ring_x + o), offd);
+          }
+          st_stream(reinterpret_cast<float4 *>(p.X + o), acc);
+          if (HAS_Z) st_stream(reinterpret_cast<float4 *>(p.Z + o), vmul(tab.inv_w[row], acc));
+        }
+      }
+      // the stage may be refilled by the async proxy once every consumer warp has released it
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(empty_bar + s);
+    }
   }
 }
 

@@ -1,0 +1,115 @@
+"""Parity at the full BASELINE sizes, in the launch configuration the benchmark times.
+
+The float64 oracle cannot run 8e8 .. 6.4e9 elements in seconds, but every column of the SGP recursion
+evolves independently of every other column, so the oracle is run on sampled column windows (first
+tile, an unaligned window in the middle, the ragged last tile) fed with the very fp32 bits the GPU
+consumed, and compared element by element there.  Whole-array invariants (sum of weights, no
+non-finite value, conserved column sums) cover the rest."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from parity_util import assert_close, graph_desc, run_oracle
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_1811_10792_b200 import build
+    build.build()
+    from paper_1811_10792_b200 import binding as b
+    return b
+
+
+@pytest.fixture(scope="module")
+def inputs():
+    from paper_1811_10792_b200 import inputs as i
+    return i
+
+
+def _windows(d):
+    mid = (d // 2) | 1                                   # odd start: not vector aligned
+    return [(0, min(d, 4096)), (mid, min(d, mid + 3001)), (max(0, d - 2056), d)]
+
+
+def _run_full(binding, inputs, w, K, ld_align=256):
+    """ld_align = 256 is the benchmark's layout (rows start on 1 KB boundaries); 1 is the dense layout."""
+    n, d = w.n, w.d
+    ld = (d + ld_align - 1) // ld_align * ld_align
+    need = 4 * n * d * (4 + w.tau) + (2 << 30)
+    free_b, _ = torch.cuda.mem_get_info()
+    if free_b < need:
+        pytest.skip(f"needs {need / 2**30:.0f} GiB of device memory, {free_b / 2**30:.0f} GiB free")
+    def matrix(fill):
+        return torch.full((n, ld), fill, dtype=torch.float32, device=DEV)[:, :d]
+    X = matrix(0.0)
+    X.copy_(inputs.initial_x(w, device=DEV))
+    M = matrix(0.0) if w.momentum != 0.0 else None
+    Z = matrix(float("nan"))
+    G = matrix(0.0)
+    W = torch.ones(n, device=DEV)
+    wins = _windows(d)
+    x0 = [X[:, a:b].cpu().numpy().copy() for a, b in wins]
+    grads = [[] for _ in wins]
+    with binding.Sgp(n, d, graph_desc(w, binding), tau=w.tau, ld=ld) as h:
+        for k in range(K):
+            inputs.gradient(w, k, G)
+            for i, (a, b) in enumerate(wins):
+                grads[i].append(G[:, a:b].cpu().numpy().copy())
+            h.step(X, W, M, G, Z, k, w.lr, w.momentum, w.weight_decay, w.nesterov)
+        torch.cuda.synchronize()
+        assert h.device_status() == 0
+        sum_w, min_w, nonfinite, _ = h.check(X, W)
+    assert abs(sum_w - n) <= 1e-4 * n and min_w > 0 and nonfinite == 0
+    assert torch.isfinite(Z).all().item()
+    for i, (a, b) in enumerate(wins):
+        ww = w.scaled(b - a, K=K)
+        st = run_oracle(ww, x0[i], grads[i], K=K)
+        assert_close(f"X[{a}:{b}]", X[:, a:b].cpu().numpy(), st.x)
+        assert_close(f"Z[{a}:{b}]", Z[:, a:b].cpu().numpy(), st.z)
+        if M is not None:
+            assert_close(f"M[{a}:{b}]", M[:, a:b].cpu().numpy(), st.u)
+        assert_close("W", W.cpu().numpy(), st.w)
+    del X, M, Z, G
+    torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("ld_align", [256, 1])
+def test_resnet50_full_size(binding, inputs, ld_align):
+    _run_full(binding, inputs, inputs.WORKLOADS["resnet50"], K=3, ld_align=ld_align)
+
+
+def test_transformer_full_size(binding, inputs):
+    _run_full(binding, inputs, inputs.WORKLOADS["transformer"], K=3)
+
+
+def test_resnet50_overlap_full_size(binding, inputs):
+    _run_full(binding, inputs, inputs.WORKLOADS["resnet50_osgp1"], K=3)
+
+
+@pytest.mark.parametrize("n,d", [(256, 10_000_000), (64, 100_000_000)])
+def test_sweep_largest_points(binding, inputs, n, d):
+    """More than 2^31 elements per array: 64-bit offsets everywhere."""
+    _run_full(binding, inputs, inputs.sweep_workload(n, d), K=2)
+
+
+def test_tau_full_size_mass_conservation(binding, inputs):
+    """With zero gradients the total mass (state + ring) of every column is conserved by the delayed mix."""
+    w = dataclasses.replace(inputs.sweep_workload(64, 3_000_001), tau=2, grad_std=0.0, momentum=0.0)
+    n, d = w.n, w.d
+    X = inputs.initial_x(w, device=DEV).contiguous()
+    Z = torch.empty_like(X)
+    G = torch.zeros_like(X)
+    W = torch.ones(n, device=DEV)
+    before = X.sum(dtype=torch.float64).item()
+    scale = X.abs().sum(dtype=torch.float64).item()
+    with binding.Sgp(n, d, graph_desc(w, binding), tau=2) as h:
+        for k in range(7):
+            h.step(X, W, None, G, Z, k, w.lr, 0.0, 0.0, True)
+        sum_w, min_w, nonfinite, total = h.check(X, W)
+    assert abs(sum_w - n) <= 1e-4 * n and nonfinite == 0
+    assert abs(total - before) <= 1e-5 * scale

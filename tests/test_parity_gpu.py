@@ -325,3 +325,42 @@ def test_invalid_step_arguments(binding, inputs):
             h.set_option("no_such_knob", 1)
         h.set_option("ctas_per_sm", 3)
         assert h.get_option("ctas_per_sm") == 3
+
+
+# ------------------------------------------------------------------ bulk-copy pipelined kernel (variant 2)
+def _tma_cases(inputs):
+    import dataclasses
+    W = inputs.WORKLOADS
+    return [
+        W["resnet50"].scaled(8200),
+        W["resnet50"].scaled(128 * 700 + 4, K=7),
+        W["transformer"].scaled(256 * 9 + 12),
+        dataclasses.replace(W["resnet50_osgp1"].scaled(4104, K=20), tau=1),
+        dataclasses.replace(W["resnet50_osgp1"].scaled(4104, K=9), tau=3),
+        inputs.sweep_workload(4, 10_000), inputs.sweep_workload(16, 10_000),
+        inputs.sweep_workload(64, 10_000), inputs.sweep_workload(256, 10_000),
+        dataclasses.replace(inputs.sweep_workload(5, 516), nesterov=False),
+        inputs.Workload("one", n=1, d=4, K=3, graph="exp", lr=0.1, momentum=0.9),
+    ]
+
+
+@pytest.mark.parametrize("case", range(11))
+@pytest.mark.parametrize("opts", [{"variant": 2}, {"variant": 2, "stages": 4, "ctas_per_sm": 1},
+                                  {"variant": 2, "stages": 3, "tile_cols": 64}, {"variant": 3},
+                                  {"variant": 3, "stages": 3, "tile_cols": 512, "ctas_per_sm": 1}])
+def test_bulk_copy_kernel_matches_oracle_and_register_kernel(binding, inputs, case, opts):
+    w = _tma_cases(inputs)[case]
+    ref = _run_gpu(binding, inputs, w, options={"variant": 1})
+    out = _run_gpu(binding, inputs, w, options=opts)
+    _compare(w, out)
+    for name in ("X", "W", "M", "Z"):
+        assert np.array_equal(ref[name], out[name], equal_nan=True), name     # same FMA order: same bits
+    if w.tau > 0:
+        assert np.array_equal(ref["ring"][0], out["ring"][0]) and np.array_equal(ref["ring"][1], out["ring"][1])
+
+
+def test_bulk_copy_kernel_with_row_pitch(binding, inputs):
+    w = inputs.sweep_workload(16, 2052)
+    for variant in (2, 3):
+        out = _run_gpu(binding, inputs, w, ld=w.d + 8, offset=4, options={"variant": variant})
+        _compare(w, out)
