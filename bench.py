@@ -32,7 +32,10 @@ NOMINAL_HBM_GBS = 8000.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused step kernel, from the ncu capture
 # summarised under profiles/ (captured on a column-scaled case and scaled by the units processed).
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    # profiles/sgp_step_tma_resnet50_small_ncu.md: 1477.7 MB per launch at d = 2,000,000, x (25,557,032 / 2,000,000)
+    "resnet50": 18.883e9,
+}
 
 
 def bytes_per_update(w, write_z=True) -> int:
@@ -166,6 +169,22 @@ def run_reference(args, w):
     print(json.dumps(line), flush=True)
 
 
+def max_over_ranks(value: float, device="cpu") -> float:
+    """Slowest rank's figure (all-reduce MAX over the default process group; identity for one rank)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(world: int, units_per_rank_per_step: int, steps: int, max_ms: float) -> float:
+    """Replicas only: every rank processes the same number of units; the job ends with the slowest rank."""
+    return world * units_per_rank_per_step * steps / (max_ms * 1e-3)
+
+
 def workload_config(w, extra=None):
     cfg = {"workload": f"{w.name}: n={w.n} nodes x d={w.d} fp32 parameters, {w.peers}-peer exponential digraph"
                        if w.graph == "exp" else f"{w.name}: n={w.n} x d={w.d}, {w.graph} digraph",
@@ -267,11 +286,8 @@ def main():
     total_ms = evs[0].elapsed_time(evs[K])
     per_step_ms = [evs[i].elapsed_time(evs[i + 1]) for i in range(K)]
     assert h.device_status() == 0
-    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    max_ms = float(t.item())
-    value = world * n * d * K / (max_ms * 1e-3)
+    max_ms = max_over_ranks(total_ms, dev)
+    value = whole_job_value(world, n * d, K, max_ms)
 
     # ---- end to end through the host-buffer entry point (gradients in, de-biased parameters out)
     e2e = None
@@ -290,12 +306,10 @@ def main():
             h.step_host(X, Wt, M, hG, hZ, dG, Z, Wm + K + 1 + i, w.lr, w.momentum, w.weight_decay, w.nesterov)
         torch.cuda.synchronize()
         dt = time.perf_counter() - t0
-        t2 = torch.tensor([dt], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(t2, op=dist.ReduceOp.MAX)
-        e2e = {"value": world * n * d * e2e_steps / float(t2.item()), "unit": UNIT,
+        dt_max = max_over_ranks(dt, dev)
+        e2e = {"value": whole_job_value(world, n * d, e2e_steps, dt_max * 1e3), "unit": UNIT,
                "h2d_bytes_per_step": arr_bytes, "d2h_bytes_per_step": arr_bytes, "steps": e2e_steps,
-               "ms_per_step": float(t2.item()) * 1e3 / e2e_steps}
+               "ms_per_step": dt_max * 1e3 / e2e_steps}
         del hG, hZ
     sampler.stop()
 
