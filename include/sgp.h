@@ -172,6 +172,36 @@ int sgp_check(sgp_handle *h, const float *d_X, const float *d_W, double *h_stats
 int sgp_set_option(sgp_handle *h, const char *key, int64_t value);
 int sgp_get_option(const sgp_handle *h, const char *key, int64_t *value);
 
+/*
+ * sgp_step_static: the tau = 0 fused step of sgp_step for callers that cannot allocate device memory.
+ * (The paper has no counterpart: this entry point exists for deployment reasons only.)
+ *
+ * Who needs it: a process whose device memory was handed, whole, to a framework's pool at start-up; a
+ * latency-critical loop that cannot afford the device-wide synchronisation an allocation implies; a
+ * plug-in running under a memory-accounting wrapper.  sgp_create allocates, so these callers use no
+ * handle.  This call performs no cudaMalloc/cudaFree and calls no allocating library routine: the
+ * step's in-neighbour table and its two launch words live in one file-scope device array inside the
+ * library image (about 40 KB, held by every GPU that loads the library until the process exits).
+ *
+ * The mixing matrix of the step is passed as HOST arrays in the CSR form sgp_schedule_get produces
+ * (h_rowptr[n+1], h_col[nnz], h_val[nnz]; the host-only schedule compiler needs no GPU).  Limits:
+ * n <= SGP_MAX_NODES and nnz <= SGP_STATIC_MAX_NNZ, otherwise SGP_ERR_ARG ("use a handle"); a table
+ * whose row pointers or column indices are inconsistent returns SGP_ERR_GRAPH.  X, W, M are updated
+ * in place, G is read, Z (may be NULL) is written, exactly as by sgp_step; M may be NULL when
+ * momentum == 0.  Asynchronous on `stream`.
+ *
+ * Set-up: the first call made with a given device current resolves the device address of the static
+ * array (cudaGetSymbolAddress) and caches it for that device; make that first call outside any stream
+ * capture.  Sharing: all calls on a device use the same array, and it keeps the last call's
+ * contents; every call rewrites the table and clears the launch words in stream order, so calls
+ * issued to ONE stream are safe back to back, while calls that may overlap on the GPU (different
+ * streams without a dependency) race and must not be made.
+ */
+#define SGP_STATIC_MAX_NNZ 4096
+int sgp_step_static(int n, int64_t d, int64_t ld, const int32_t *h_rowptr, const int32_t *h_col,
+                    const float *h_val, int64_t nnz, float *d_X, float *d_W, float *d_M, const float *d_G,
+                    float *d_Z, float lr, float momentum, float weight_decay, int nesterov, void *stream);
+
 /* Reads the handle's device status word (0 = no kernel ever gave up a bounded wait).  Synchronises. */
 int sgp_device_status(sgp_handle *h, unsigned *status);
 /* cudaError_t value latched by the last call that returned SGP_ERR_CUDA on this handle (0 if none). */

@@ -16,6 +16,7 @@ LIB_PATH = os.path.join(_PKG_DIR, "libsgp.so")
 
 SGP_OK, SGP_ERR_ARG, SGP_ERR_GRAPH, SGP_ERR_CUDA, SGP_ERR_ALLOC, SGP_ERR_STATE, SGP_ERR_DEVICE = 0, -1, -2, -3, -4, -5, -6
 SGP_MAX_NODES = 256
+SGP_STATIC_MAX_NNZ = 4096
 SGP_GRAPH_EXP_PEERS, SGP_GRAPH_COMPLETE, SGP_GRAPH_RANDOM_OUTDEG, SGP_GRAPH_CUSTOM = 0, 1, 2, 3
 
 # every symbol include/sgp.h declares
@@ -23,7 +24,7 @@ EXPORTS = [
     "sgp_schedule_compile", "sgp_schedule_destroy", "sgp_schedule_period", "sgp_schedule_nnz", "sgp_schedule_get",
     "sgp_create", "sgp_destroy", "sgp_get_schedule", "sgp_step", "sgp_debias", "sgp_step_host", "sgp_reset",
     "sgp_ring_export", "sgp_ring_import", "sgp_check", "sgp_set_option", "sgp_get_option", "sgp_device_status",
-    "sgp_last_cuda_error", "sgp_strerror", "sgp_version",
+    "sgp_last_cuda_error", "sgp_strerror", "sgp_version", "sgp_step_static",
 ]
 
 
@@ -71,6 +72,7 @@ def _load() -> C.CDLL:
         "sgp_device_status": [vp, C.POINTER(C.c_uint)],
         "sgp_last_cuda_error": [vp],
         "sgp_version": [],
+        "sgp_step_static": [i32, i64, i64, vp, vp, vp, i64, vp, vp, vp, vp, vp, f32, f32, f32, i32, vp],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
@@ -280,6 +282,22 @@ class Sgp:
 
     def last_cuda_error(self) -> int:
         return _lib.sgp_last_cuda_error(self._h)
+
+
+def step_static(n: int, d: int, ld: int, rowptr, col, val, X, W, M, G, Z, lr: float, momentum: float = 0.0,
+                weight_decay: float = 0.0, nesterov: bool = True, stream=None) -> None:
+    """sgp_step_static: the tau = 0 fused step without a handle and without any device allocation.
+
+    For callers that cannot call cudaMalloc (all device memory owned by a pool, latency-critical loops).
+    rowptr / col / val are HOST numpy arrays in the form Schedule.get(k) returns (at most
+    SGP_STATIC_MAX_NNZ entries).  Calls must be ordered on one stream: they share one static device table.
+    """
+    rowptr = np.ascontiguousarray(rowptr, dtype=np.int32)
+    col = np.ascontiguousarray(col, dtype=np.int32)
+    val = np.ascontiguousarray(val, dtype=np.float32)
+    _check(_lib.sgp_step_static(n, d, ld, rowptr.ctypes.data, col.ctypes.data, val.ctypes.data, len(col), _ptr(X),
+                                _ptr(W), _ptr(M), _ptr(G), _ptr(Z), lr, momentum, weight_decay, int(bool(nesterov)),
+                                _stream_ptr(stream)), "sgp_step_static")
 
 
 def version() -> int:

@@ -10,7 +10,7 @@ ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libsgp.so")
 
-SOURCES = ["sgp_api.cu", "schedule.cpp"]
+SOURCES = ["sgp_api.cu", "sgp_static.cu", "schedule.cpp"]
 HEADERS = ["step_kernels.cuh", "aux_kernels.cuh", "schedule.h"]
 
 NVCC_FLAGS = [
