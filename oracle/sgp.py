@@ -15,6 +15,10 @@ Readings fixed here where the paper leaves a choice:
   * K steps means k = 0 .. K-1; u^(0) = 0; w^(0) = 1; z^(0) = x^(0).
   * Weight decay adds lambda * x (the biased numerator the optimiser steps on,
     App. C description of the compute thread) to the gradient.
+  * Adam: the paper combines SGP with "the Adam preconditioner" for its Transformer runs (Sec. 6.2,
+    App. C.1) without a listing.  Reading: the bias-corrected Adam step of Kingma & Ba replaces
+    Alg. 3 lines 4-5 (gradient taken at z, step applied to the numerator x, both moment vectors local
+    to a node and never gossiped); weight decay is added to the gradient as for SGD.
   * Delay tau: the self term p_ii h_i is never delayed; every other message
     (p_ij h_j, p_ij w_j) sent at step k is added at step k + tau, i.e. it lands
     in x^(k+tau+1); messages are sent every step; both parts accumulate;
@@ -37,6 +41,7 @@ class SGPState:
     w: np.ndarray                      # n push-sum weights
     u: np.ndarray                      # n x d momentum buffers
     z: np.ndarray                      # n x d de-biased parameters
+    v: np.ndarray = None               # n x d Adam second moments (u holds the first moments)
     transit_x: deque = field(default_factory=deque)   # tau in-flight (n x d) messages, oldest first
     transit_w: deque = field(default_factory=deque)   # tau in-flight (n) weight messages
 
@@ -45,7 +50,7 @@ def init_state(x0, tau: int = 0) -> SGPState:
     """Alg. 1 'Require' line: w = 1, z = x; Alg. 3: u = 0; virtual nodes hold 0."""
     x = np.array(x0, dtype=np.float64)
     n, d = x.shape
-    st = SGPState(x=x, w=np.ones(n), u=np.zeros((n, d)), z=x.copy())
+    st = SGPState(x=x, w=np.ones(n), u=np.zeros((n, d)), z=x.copy(), v=np.zeros((n, d)))
     for _ in range(tau):
         st.transit_x.append(np.zeros((n, d)))
         st.transit_w.append(np.zeros(n))
@@ -73,6 +78,22 @@ def local_update(x, u, g, lr, momentum=0.0, nesterov=True, weight_decay=0.0):
     return h, u_next
 
 
+def local_update_adam(x, m, v, g, t, lr, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0):
+    """Half step with the Adam preconditioner; t = 1, 2, ... counts the steps taken including this one.
+
+    Returns (h, m_next, v_next).
+    """
+    g = np.asarray(g, dtype=np.float64)
+    if weight_decay != 0.0:
+        g = g + weight_decay * x
+    m_next = beta1 * m + (1.0 - beta1) * g
+    v_next = beta2 * v + (1.0 - beta2) * g * g
+    m_hat = m_next / (1.0 - beta1 ** t)
+    v_hat = v_next / (1.0 - beta2 ** t)
+    h = x - lr * m_hat / (np.sqrt(v_hat) + eps)
+    return h, m_next, v_next
+
+
 def mix(P, h, w):
     """One PushSum iteration, no delay (Alg. 1 lines 6-7): x' = P h, w' = P w."""
     return P @ h, P @ w
@@ -96,9 +117,16 @@ def mix_delayed(P, h, w, transit_x, transit_w):
     return x_next, w_next
 
 
-def sgp_step(st: SGPState, g, P, lr, momentum=0.0, nesterov=True, weight_decay=0.0) -> SGPState:
-    """One full SGP iteration in place on ``st`` (gradient g was taken at st.z)."""
-    h, st.u = local_update(st.x, st.u, g, lr, momentum, nesterov, weight_decay)
+def sgp_step(st: SGPState, g, P, lr, momentum=0.0, nesterov=True, weight_decay=0.0, adam=None) -> SGPState:
+    """One full SGP iteration in place on ``st`` (gradient g was taken at st.z).
+
+    ``adam`` = (t, beta1, beta2, eps) switches the local update to Adam.
+    """
+    if adam is None:
+        h, st.u = local_update(st.x, st.u, g, lr, momentum, nesterov, weight_decay)
+    else:
+        t, beta1, beta2, eps = adam
+        h, st.u, st.v = local_update_adam(st.x, st.u, st.v, g, t, lr, beta1, beta2, eps, weight_decay)
     if len(st.transit_x) == 0:
         st.x, st.w = mix(P, h, st.w)
     else:
@@ -108,17 +136,19 @@ def sgp_step(st: SGPState, g, P, lr, momentum=0.0, nesterov=True, weight_decay=0
 
 
 def sgp_run(x0, K, P_of_k, grad_of_k, lr, momentum=0.0, nesterov=True, weight_decay=0.0,
-            tau=0, history=None) -> SGPState:
+            tau=0, history=None, adam=None) -> SGPState:
     """K iterations k = 0 .. K-1.
 
     ``P_of_k(k)`` returns the dense mixing matrix of step k; ``grad_of_k(k, z)``
     returns the n x d stochastic gradients evaluated at the de-biased ``z``.
     If ``history`` is a list, a snapshot (x, w, u, z) is appended after every step.
+    ``adam`` = (beta1, beta2, eps) runs Adam-SGP (step count t = k + 1).
     """
     st = init_state(x0, tau)
     for k in range(K):
         g = grad_of_k(k, st.z)
-        sgp_step(st, g, P_of_k(k), lr, momentum, nesterov, weight_decay)
+        sgp_step(st, g, P_of_k(k), lr, momentum, nesterov, weight_decay,
+                 adam=None if adam is None else (k + 1, *adam))
         if history is not None:
             history.append((st.x.copy(), st.w.copy(), st.u.copy(), st.z.copy()))
     return st

@@ -257,3 +257,47 @@ def test_tau_zero_equals_no_transit():
 def test_debias_helper():
     x = np.arange(6, dtype=float).reshape(2, 3)
     assert np.array_equal(O.debias(x, [2.0, 0.5]), [[0, 0.5, 1.0], [6, 8, 10]])
+
+
+# ---------------------------------------------------------------- Adam-SGP
+@pytest.mark.parametrize("wd", [0.0, 1e-2])
+def test_single_node_adam_matches_torch_adam(wd):
+    # n = 1, P = [1]: the Adam half step must be the library's Adam (bias correction, eps outside the sqrt)
+    d, K, lr, b1, b2, eps = 9, 25, 1e-2, 0.9, 0.98, 1e-8
+    rng = np.random.default_rng(50)
+    x0 = rng.standard_normal((1, d))
+    G, gfun = _rand_grads(1, d, K, 51)
+    st = O.sgp_run(x0, K, lambda k: np.ones((1, 1)), gfun, lr, weight_decay=wd, adam=(b1, b2, eps))
+    p = torch.tensor(x0[0].copy(), dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.Adam([p], lr=lr, betas=(b1, b2), eps=eps, weight_decay=wd)
+    for k in range(K):
+        p.grad = torch.tensor(G[k, 0].copy(), dtype=torch.float64)
+        opt.step()
+    assert np.allclose(st.x[0], p.detach().numpy(), rtol=1e-11, atol=1e-13)
+    assert np.allclose(st.u[0], opt.state[p]["exp_avg"].numpy(), rtol=1e-12, atol=1e-14)
+    assert np.allclose(st.v[0], opt.state[p]["exp_avg_sq"].numpy(), rtol=1e-12, atol=1e-16)
+
+
+def test_adam_first_step_by_hand():
+    # t = 1: m_hat = g, v_hat = g^2  =>  h = x - lr * g / (|g| + eps) = x - lr * sign(g) (up to eps)
+    x0 = np.array([[1.0, -2.0, 0.5]])
+    g = np.array([[0.3, -4.0, 1e-3]])
+    st = O.sgp_run(x0, 1, lambda k: np.ones((1, 1)), lambda k, z: g, 0.1, adam=(0.9, 0.999, 1e-12))
+    assert np.allclose(st.x, x0 - 0.1 * np.sign(g), rtol=0, atol=1e-9)
+    assert np.allclose(st.u, 0.1 * g) and np.allclose(st.v, 1e-3 * g * g)
+
+
+def test_adam_sgp_moments_stay_local_and_mass_is_mixed():
+    n, d, K = 8, 5, 6
+    rng = np.random.default_rng(52)
+    x0 = rng.standard_normal((n, d))
+    G, gfun = _rand_grads(n, d, K, 53)
+    Pk = lambda k: S.mixing_matrix("random", n, k, seed=9, max_outdeg=3, num_steps=5)
+    st = O.sgp_run(x0, K, Pk, gfun, 1e-2, adam=(0.9, 0.99, 1e-8), tau=1)
+    m = np.zeros((n, d)); v = np.zeros((n, d))
+    for k in range(K):
+        m = 0.9 * m + 0.1 * G[k]
+        v = 0.99 * v + 0.01 * G[k] ** 2
+    assert np.allclose(st.u, m, rtol=1e-13) and np.allclose(st.v, v, rtol=1e-13)     # independent of the graph
+    _, sw = O.total_mass(st)
+    assert abs(sw - n) < 1e-12
