@@ -41,7 +41,9 @@ NCU_TRAFFIC_BYTES = {
 def bytes_per_update(w, write_z=True) -> int:
     """Algorithmic HBM bytes per node-parameter per step (fp32, in place)."""
     b = 4 * (2 + 1)                       # read x, g; write x
-    if w.momentum != 0.0:
+    if getattr(w, "optimizer", "sgd") == "adam":
+        b += 16                           # read and write both moment arrays
+    elif w.momentum != 0.0:
         b += 8                            # read u, write u
     if write_z:
         b += 4
@@ -133,12 +135,13 @@ def oracle_sample_run(w, sample_cols: int, steps: int, warmup: int):
     G = torch.empty((w.n, sample_cols), dtype=torch.float32)
     grads = [inputs.gradient(w, k, G).numpy().astype(np.float64) for k in range(min(4, steps + warmup))]
     P_of_k = oracle_P_of_k(w)
+    adam = (lambda k: (k + 1, w.beta1, w.beta2, w.adam_eps)) if w.optimizer == "adam" else (lambda k: None)
     st = osgp.init_state(x0, w.tau)
     for k in range(warmup):
-        osgp.sgp_step(st, grads[k % len(grads)], P_of_k(k), w.lr, w.momentum, w.nesterov, w.weight_decay)
+        osgp.sgp_step(st, grads[k % len(grads)], P_of_k(k), w.lr, w.momentum, w.nesterov, w.weight_decay, adam=adam(k))
     t0 = time.perf_counter()
     for k in range(warmup, warmup + steps):
-        osgp.sgp_step(st, grads[k % len(grads)], P_of_k(k), w.lr, w.momentum, w.nesterov, w.weight_decay)
+        osgp.sgp_step(st, grads[k % len(grads)], P_of_k(k), w.lr, w.momentum, w.nesterov, w.weight_decay, adam=adam(k))
     dt = (time.perf_counter() - t0) / steps
     threads = 1
     try:
@@ -189,8 +192,9 @@ def workload_config(w, extra=None):
     cfg = {"workload": f"{w.name}: n={w.n} nodes x d={w.d} fp32 parameters, {w.peers}-peer exponential digraph"
                        if w.graph == "exp" else f"{w.name}: n={w.n} x d={w.d}, {w.graph} digraph",
            "n": w.n, "d": w.d, "graph": w.graph, "peers": w.peers, "tau": w.tau, "lr": w.lr, "momentum": w.momentum,
-           "nesterov": w.nesterov, "weight_decay": w.weight_decay, "writes_z": True,
-           "l2_policy": "inputs larger than L2 (every array >= 3 GB, streamed once per step)"}
+           "nesterov": w.nesterov, "weight_decay": w.weight_decay, "writes_z": True, "optimizer": w.optimizer,
+           "l2_policy": ("inputs larger than L2 (arrays of %.2f GB each, streamed once per step)" % (4e-9 * w.n * w.d))
+                        if 4 * w.n * w.d > (512 << 20) else "working set comparable to L2: a launch-latency figure"}
     if extra:
         cfg.update(extra)
     return cfg
@@ -201,7 +205,8 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="resnet50")
+    ap.add_argument("--workload", default="resnet50",
+                    help="resnet50 | transformer | resnet50_osgp1 | tiny | sweep:<n>:<d>")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--d", type=int, default=0, help="override the parameter count (profiling on a small case)")
     ap.add_argument("--no-e2e", action="store_true")
@@ -213,7 +218,11 @@ def main():
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
     from paper_1811_10792_b200 import inputs
-    w = inputs.WORKLOADS[args.workload]
+    if args.workload.startswith("sweep:"):            # sweep:<n>:<d>  (scaling-sweep point, random digraphs)
+        _, sn, sd = args.workload.split(":")
+        w = inputs.sweep_workload(int(sn), int(sd))
+    else:
+        w = inputs.WORKLOADS[args.workload]
     if args.d > 0:
         w = w.scaled(args.d)
     if args.impl == "reference":
@@ -239,7 +248,7 @@ def main():
     n, d, K, Wm = w.n, w.d, args.steps, args.warmup
     free_b, _total_b = torch.cuda.mem_get_info()
     arr_bytes = 4 * n * d
-    n_state = 3 + (1 if w.tau else 0)                       # X, M, Z (+ ring inside the handle)
+    n_state = 3 + (1 if w.tau else 0) + (1 if w.optimizer == "adam" else 0)   # X, M, Z (+ ring, + second moment)
     pool = max(1, min(K, int((free_b * 0.6 - n_state * arr_bytes) // arr_bytes)))
     ld = (d + args.ld_align - 1) // args.ld_align * args.ld_align
 
@@ -249,7 +258,9 @@ def main():
 
     X = matrix()
     X.copy_(inputs.initial_x(w, device=dev))
-    M = matrix() if w.momentum != 0.0 else None
+    adam = w.optimizer == "adam"
+    M = matrix() if (w.momentum != 0.0 or adam) else None
+    V2 = matrix() if adam else None
     Z = matrix()
     Wt = torch.ones(n, device=dev)
     Gs = []
@@ -263,7 +274,10 @@ def main():
         h.set_option(key, int(val))
 
     def step(k):
-        h.step(X, Wt, M, Gs[k % pool], Z, k, w.lr, w.momentum, w.weight_decay, w.nesterov)
+        if adam:
+            h.step_adam(X, Wt, M, V2, Gs[k % pool], Z, k, k + 1, w.lr, w.beta1, w.beta2, w.adam_eps, w.weight_decay)
+        else:
+            h.step(X, Wt, M, Gs[k % pool], Z, k, w.lr, w.momentum, w.weight_decay, w.nesterov)
 
     sampler = ClockSampler(local_rank)
     sampler.start()
@@ -291,7 +305,7 @@ def main():
 
     # ---- end to end through the host-buffer entry point (gradients in, de-biased parameters out)
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not adam:
         hG = torch.empty((n, ld), dtype=torch.float32, pin_memory=True)[:, :d]
         hZ = torch.empty((n, ld), dtype=torch.float32, pin_memory=True)[:, :d]
         hG.copy_(Gs[0])

@@ -131,6 +131,23 @@ int sgp_get_schedule(const sgp_handle *h, const sgp_schedule **s);
 int sgp_step(sgp_handle *h, float *d_X, float *d_W, float *d_M, const float *d_G, float *d_Z,
              int64_t k, float lr, float momentum, float weight_decay, int nesterov, void *stream);
 
+/*
+ * sgp_step_adam: the same iteration with the Adam preconditioner in place of the momentum update
+ * (Sec. 6.2 and App. C.1: SGP combined with Adam for the Transformer runs; the paper prints no listing,
+ * so the update is the standard bias-corrected Adam applied to the numerator with the gradient taken
+ * at Z, moments local to each node and never mixed):
+ *     g~ = G + weight_decay * X
+ *     M1 <- beta1*M1 + (1-beta1) g~ ;  M2 <- beta2*M2 + (1-beta2) g~^2
+ *     h  = X - lr/(1-beta1^t) * M1 / ( sqrt(M2)/sqrt(1-beta2^t) + eps )
+ * followed by the mix, weight update and de-bias of sgp_step (any tau).  t >= 1 is the 1-based count
+ * of Adam steps taken so far including this one; k >= 0 selects the schedule and ring slots.
+ * M1, M2 are n x ld fp32 device arrays updated in place (start at zero).  32 bytes of HBM traffic per
+ * node-parameter with Z written.
+ */
+int sgp_step_adam(sgp_handle *h, float *d_X, float *d_W, float *d_M1, float *d_M2, const float *d_G, float *d_Z,
+                  int64_t k, int64_t t, float lr, float beta1, float beta2, float eps, float weight_decay,
+                  void *stream);
+
 /* sgp_debias: Z_i = X_i * (1 / W_i) for all nodes (Alg. 1 line 8), one pass.  X may equal Z. */
 int sgp_debias(sgp_handle *h, const float *d_X, const float *d_W, float *d_Z, void *stream);
 
@@ -167,6 +184,8 @@ int sgp_check(sgp_handle *h, const float *d_X, const float *d_W, double *h_stats
  *   "tile_cols"    columns per tile (multiple of 4; 0 = automatic)
  *   "ctas_per_sm"  persistent CTAs per SM (0 = automatic)
  *   "stages"       shared-memory stages of the bulk-copy pipeline (0 = automatic, at most 8)
+ * Read-only through sgp_get_option: "last_variant", "last_grid", "last_smem", "last_tile_cols" describe
+ * the most recent step launch of the handle (which kernel ran, CTAs, dynamic shared memory, tile width).
  * Unknown keys or unsupported values return SGP_ERR_ARG and change nothing.
  */
 int sgp_set_option(sgp_handle *h, const char *key, int64_t value);

@@ -25,6 +25,7 @@ EXPORTS = [
     "sgp_create", "sgp_destroy", "sgp_get_schedule", "sgp_step", "sgp_debias", "sgp_step_host", "sgp_reset",
     "sgp_ring_export", "sgp_ring_import", "sgp_check", "sgp_set_option", "sgp_get_option", "sgp_device_status",
     "sgp_last_cuda_error", "sgp_strerror", "sgp_version", "sgp_step_static",
+    "sgp_step_adam",
 ]
 
 
@@ -62,6 +63,7 @@ def _load() -> C.CDLL:
         "sgp_get_schedule": [vp, C.POINTER(vp)],
         "sgp_step": [vp, vp, vp, vp, vp, vp, i64, f32, f32, f32, i32, vp],
         "sgp_debias": [vp, vp, vp, vp, vp],
+        "sgp_step_adam": [vp, vp, vp, vp, vp, vp, vp, i64, i64, f32, f32, f32, f32, f32, vp],
         "sgp_step_host": [vp, vp, vp, vp, vp, vp, vp, vp, i64, f32, f32, f32, i32, i64],
         "sgp_reset": [vp, vp],
         "sgp_ring_export": [vp, vp, vp, vp],
@@ -240,6 +242,14 @@ class Sgp:
         self._check_mat(Z, "Z", allow_none=True)
         _check(_lib.sgp_step(self._h, _ptr(X), _ptr(W), _ptr(M), _ptr(G), _ptr(Z), k, lr, momentum, weight_decay,
                              int(bool(nesterov)), _stream_ptr(stream)), "sgp_step")
+
+    def step_adam(self, X, W, M1, M2, G, Z, k: int, t: int, lr: float, beta1: float = 0.9, beta2: float = 0.999,
+                  eps: float = 1e-8, weight_decay: float = 0.0, stream=None) -> None:
+        for name, m in (("X", X), ("M1", M1), ("M2", M2), ("G", G)):
+            self._check_mat(m, name)
+        self._check_mat(Z, "Z", allow_none=True)
+        _check(_lib.sgp_step_adam(self._h, _ptr(X), _ptr(W), _ptr(M1), _ptr(M2), _ptr(G), _ptr(Z), k, t, lr, beta1,
+                                  beta2, eps, weight_decay, _stream_ptr(stream)), "sgp_step_adam")
 
     def debias(self, X, W, Z, stream=None) -> None:
         self._check_mat(X, "X")

@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <cmath>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -36,6 +37,7 @@ struct sgp_handle {
   unsigned *d_words = nullptr;  // [0] ticket, [1] status
   double *d_stats = nullptr;    // 4 doubles for sgp_check
   int64_t opt_variant = 0, opt_tile_cols = 0, opt_ctas_per_sm = 0, opt_stages = 0;
+  int64_t last_variant = 0, last_grid = 0, last_smem = 0, last_tile_cols = 0;   // of the most recent step launch
   cudaStream_t s_h2d = nullptr, s_compute = nullptr, s_d2h = nullptr;
   std::vector<cudaEvent_t> ev_in, ev_done;
   int last_cuda_error = 0;
@@ -90,33 +92,35 @@ void free_handle(sgp_handle *h) {
 
 using StepKernel = void (*)(const StepParams, const ConstTable);
 
-template <int VEC, bool HAS_M, bool NESTEROV, bool HAS_Z>
-StepKernel pick_ring(bool has_ring) {
-  return has_ring ? sgp::sgp_step_regs_kernel<VEC, HAS_M, NESTEROV, HAS_Z, true>
-                  : sgp::sgp_step_regs_kernel<VEC, HAS_M, NESTEROV, HAS_Z, false>;
-}
-template <int VEC, bool HAS_M, bool NESTEROV>
-StepKernel pick_z(bool has_z, bool has_ring) {
-  return has_z ? pick_ring<VEC, HAS_M, NESTEROV, true>(has_ring) : pick_ring<VEC, HAS_M, NESTEROV, false>(has_ring);
+template <int VEC, int UPD>
+StepKernel pick_regs_flags(bool has_z, bool has_ring) {
+  if (has_z) return has_ring ? sgp::sgp_step_regs_kernel<VEC, UPD, true, true> : sgp::sgp_step_regs_kernel<VEC, UPD, true, false>;
+  return has_ring ? sgp::sgp_step_regs_kernel<VEC, UPD, false, true> : sgp::sgp_step_regs_kernel<VEC, UPD, false, false>;
 }
 template <int VEC>
-StepKernel pick_update(bool has_m, bool nesterov, bool has_z, bool has_ring) {
-  if (!has_m) return pick_z<VEC, false, false>(has_z, has_ring);
-  return nesterov ? pick_z<VEC, true, true>(has_z, has_ring) : pick_z<VEC, true, false>(has_z, has_ring);
+StepKernel pick_regs(int upd, bool has_z, bool has_ring) {
+  switch (upd) {
+    case sgp::kUpdSgd: return pick_regs_flags<VEC, sgp::kUpdSgd>(has_z, has_ring);
+    case sgp::kUpdHeavyBall: return pick_regs_flags<VEC, sgp::kUpdHeavyBall>(has_z, has_ring);
+    case sgp::kUpdNesterov: return pick_regs_flags<VEC, sgp::kUpdNesterov>(has_z, has_ring);
+    default: return pick_regs_flags<VEC, sgp::kUpdAdam>(has_z, has_ring);
+  }
 }
 
 using TmaKernel = void (*)(const StepParams, const ConstTable, const sgp::TmaMaps, const int, const int);
 
-template <bool HAS_M, bool NESTEROV>
-TmaKernel pick_tma_z(bool has_z, bool has_ring) {
-  if (has_z) return has_ring ? sgp::sgp_step_tma_kernel<HAS_M, NESTEROV, true, true>
-                             : sgp::sgp_step_tma_kernel<HAS_M, NESTEROV, true, false>;
-  return has_ring ? sgp::sgp_step_tma_kernel<HAS_M, NESTEROV, false, true>
-                  : sgp::sgp_step_tma_kernel<HAS_M, NESTEROV, false, false>;
+template <int UPD>
+TmaKernel pick_tma_flags(bool has_z, bool has_ring) {
+  if (has_z) return has_ring ? sgp::sgp_step_tma_kernel<UPD, true, true> : sgp::sgp_step_tma_kernel<UPD, true, false>;
+  return has_ring ? sgp::sgp_step_tma_kernel<UPD, false, true> : sgp::sgp_step_tma_kernel<UPD, false, false>;
 }
-TmaKernel pick_tma(bool has_m, bool nesterov, bool has_z, bool has_ring) {
-  if (!has_m) return pick_tma_z<false, false>(has_z, has_ring);
-  return nesterov ? pick_tma_z<true, true>(has_z, has_ring) : pick_tma_z<true, false>(has_z, has_ring);
+TmaKernel pick_tma(int upd, bool has_z, bool has_ring) {
+  switch (upd) {
+    case sgp::kUpdSgd: return pick_tma_flags<sgp::kUpdSgd>(has_z, has_ring);
+    case sgp::kUpdHeavyBall: return pick_tma_flags<sgp::kUpdHeavyBall>(has_z, has_ring);
+    case sgp::kUpdNesterov: return pick_tma_flags<sgp::kUpdNesterov>(has_z, has_ring);
+    default: return pick_tma_flags<sgp::kUpdAdam>(has_z, has_ring);
+  }
 }
 
 struct StepArgs {
@@ -125,8 +129,15 @@ struct StepArgs {
   float *Z;
   int64_t k;
   float lr, momentum, wd;
-  int nesterov;
+  int upd;                 // sgp::kUpd*
+  float *V = nullptr;      // Adam second moment
+  float beta1 = 0.f, beta2 = 0.f, eps = 0.f, adam_step = 0.f, adam_rsqrt_bc2 = 0.f;
 };
+
+inline int update_kind(float momentum, int nesterov) {
+  if (momentum == 0.0f) return sgp::kUpdSgd;
+  return nesterov != 0 ? sgp::kUpdNesterov : sgp::kUpdHeavyBall;
+}
 
 // Fills the launch-independent part of the kernel arguments for step a.k.
 void fill_params(const sgp_handle *h, const StepArgs &a, int64_t c0, int64_t c1, bool update_w, StepParams *out) {
@@ -136,8 +147,14 @@ void fill_params(const sgp_handle *h, const StepArgs &a, int64_t c0, int64_t c1,
   p.X = a.X;
   p.W = a.W;
   p.M = a.M;
+  p.V = a.V;
   p.G = a.G;
   p.Z = a.Z;
+  p.beta1 = a.beta1;
+  p.beta2 = a.beta2;
+  p.eps = a.eps;
+  p.adam_step = a.adam_step;
+  p.adam_rsqrt_bc2 = a.adam_rsqrt_bc2;
   if (h->tau > 0) {
     const int64_t rs = a.k % h->tau;
     p.ring_x = h->ring_x + rs * h->n * h->ld;
@@ -173,7 +190,7 @@ size_t table_smem_bytes(const sgp_handle *h, int nnz) { return (static_cast<size
 // Heuristics from measurements on B200.  The step is HBM-bound; what decides the achieved bandwidth
 // is the length of the contiguous row segments (>= 1 KB), the bytes in flight per SM and a grid that
 // is exactly one wave.  Measured (fraction of the copy bandwidth, rows on 1 KB boundaries):
-//   momentum, n <= 16 : register-staged 0.97, TMA 0.90      momentum, n = 32 : TMA 0.97, register-staged 0.95
+//   momentum, n <= 24 : register-staged 0.97, TMA 0.90      momentum, n = 32 : TMA 0.97, register-staged 0.95
 //   no momentum, n=16 : TMA 0.96, register-staged 0.87      tau = 1, n = 32  : register-staged 0.97
 // cps = 0 means "as many CTAs per SM as are resident" (asked of the occupancy calculator at launch).
 // Explicit options override each field.
@@ -186,13 +203,16 @@ Plan make_plan(const sgp_handle *h, int arrays, bool has_m, int nnz, bool vec) {
     const size_t half_sm = 112 * 1024, full_sm = 224 * 1024;
     if (!has_m && 2 * per_kb + fixed <= half_sm) {
       pl = Plan{3, 256, 2, 2};
-    } else if (has_m && h->n > 16 && 2 * per_kb + fixed <= full_sm) {
+    } else if (has_m && per_kb >= 84 * 1024 && 2 * per_kb + fixed <= full_sm) {
       pl = Plan{3, 256, 2, 2 * per_kb + fixed <= half_sm ? 2 : 1};
     } else {
-      // register-staged: 1 KB row segments, or about 1024 vector items per tile when n is small;
+      // register-staged: at least 1 KB row segments and about 2048 vector items per tile;
       // the double-buffered exchange tile is 2 x n x tile_cols x 4 bytes
-      pl.tile_cols = std::max<int64_t>(256, int64_t{4} << floor_log2(std::max<int64_t>(1, 1024 / h->n)));
-      while (pl.tile_cols > 32 && 2 * static_cast<size_t>(h->n) * pl.tile_cols * 4 + fixed > 100 * 1024) pl.tile_cols >>= 1;
+      pl.tile_cols = std::max<int64_t>(256, int64_t{4} << floor_log2(std::max<int64_t>(1, 2048 / h->n)));
+      // keep the two resident CTAs' shared memory near half of the SM's 256 KB: the rest is the L1 that
+      // tracks the loads in flight (measured: n = 48 at 2 x 100 KB reaches 0.74, at 2 x 50 KB 0.93)
+      const size_t copies = h->n > 128 ? 1 : 2;
+      while (pl.tile_cols > 32 && copies * static_cast<size_t>(h->n) * pl.tile_cols * 4 + fixed > 80 * 1024) pl.tile_cols >>= 1;
     }
   }
   if (h->opt_variant > 0) pl.variant = static_cast<int>(h->opt_variant);
@@ -212,40 +232,51 @@ int launch_regs(sgp_handle *h, const StepArgs &a, const Plan &pl, int64_t c0, in
   // tile width: about kThreads * kItemsPerThread items per tile, at least 128 bytes per row segment
   const int64_t ncols = c1 - c0;
   const int min_tv = vec == 4 ? 8 : 32;
-  int64_t tv = int64_t{1} << floor_log2(std::max<int64_t>(1, sgp::kThreads * sgp::kItemsPerThread / h->n));
+  int64_t tv = int64_t{1} << floor_log2(std::max<int64_t>(1, sgp::kThreads * 4 / h->n));
   if (pl.tile_cols > 0) tv = int64_t{1} << floor_log2(std::max<int64_t>(1, pl.tile_cols / vec));
   tv = std::max<int64_t>(tv, min_tv);
   const size_t table_bytes = table_smem_bytes(h, p.nnz);
   if (h->const_ok[static_cast<size_t>(slot)]) p.table_mode = 0;
   else p.table_mode = table_bytes <= 40 * 1024 ? 1 : 2;
+  // large n: one exchange tile (two barriers per tile) so that the row segments can stay twice as long
+  p.single_buffer = h->n > 128 ? 1 : 0;
   size_t smem = 0;
   for (;;) {
-    smem = 2 * static_cast<size_t>(h->n) * tv * vec * 4 + 3 * static_cast<size_t>(h->n) * 4 +
+    smem = (p.single_buffer ? 1 : 2) * static_cast<size_t>(h->n) * tv * vec * 4 + 3 * static_cast<size_t>(h->n) * 4 +
            (p.table_mode < 2 ? table_bytes : 0);
-    if (smem <= 100 * 1024 || tv <= min_tv) break;
+    if (smem <= 110 * 1024 || tv <= min_tv) break;
     tv >>= 1;
   }
   if (smem > static_cast<size_t>(h->smem_optin)) return SGP_ERR_ARG;
   p.log2_tile_vecs = floor_log2(tv);
   const int64_t tile_cols = tv * vec;
   const int64_t ntiles = (ncols + tile_cols - 1) / tile_cols;
-  const bool has_m = a.momentum != 0.0f;
-  StepKernel kern = vec == 4 ? pick_update<4>(has_m, a.nesterov != 0, a.Z != nullptr, h->tau > 0)
-                             : pick_update<1>(has_m, a.nesterov != 0, a.Z != nullptr, h->tau > 0);
+  StepKernel kern = vec == 4 ? pick_regs<4>(a.upd, a.Z != nullptr, h->tau > 0)
+                             : pick_regs<1>(a.upd, a.Z != nullptr, h->tau > 0);
   if (smem > 48 * 1024)
     SGP_CUDA_TRY(h, cudaFuncSetAttribute(reinterpret_cast<const void *>(kern),
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
   int cps = pl.cps;
-  if (cps <= 0) {   // persistent grid of exactly one wave
-    SGP_CUDA_TRY(h, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&cps, reinterpret_cast<const void *>(kern),
-                                                                  sgp::kThreads, smem));
-    cps = std::max(1, cps);
+  if (cps <= 0) {
+    // Persistent grid of exactly one wave: CTAs resident per SM by registers, shared memory and threads.
+    // (Computed here rather than asked of the occupancy calculator, whose answer depends on the
+    // shared-memory carve-out it assumes; the hardware picks the carve-out that fits the launch.)
+    cudaFuncAttributes fa;
+    SGP_CUDA_TRY(h, cudaFuncGetAttributes(&fa, reinterpret_cast<const void *>(kern)));
+    const int regs_per_cta = ((fa.numRegs + 7) / 8 * 8) * sgp::kThreads;
+    const int by_regs = regs_per_cta > 0 ? 65536 / regs_per_cta : 8;
+    const int by_smem = static_cast<int>((227 * 1024) / (smem + fa.sharedSizeBytes + 1024));
+    cps = std::max(1, std::min({by_regs, by_smem, 2048 / sgp::kThreads}));
   }
   const int64_t grid = std::min<int64_t>(ntiles, static_cast<int64_t>(h->sm_count) * cps);
   static const ConstTable kEmptyTable{};
   const ConstTable &ct = p.table_mode == 0 ? h->const_tables[static_cast<size_t>(slot)] : kEmptyTable;
   kern<<<static_cast<unsigned>(grid), sgp::kThreads, smem, stream>>>(p, ct);
   SGP_CUDA_TRY(h, cudaGetLastError());
+  h->last_variant = 1;
+  h->last_grid = grid;
+  h->last_smem = static_cast<int64_t>(smem);
+  h->last_tile_cols = tile_cols;
   return SGP_OK;
 }
 
@@ -296,8 +327,8 @@ int launch_tma(sgp_handle *h, const StepArgs &a, const Plan &pl, int64_t c0, int
   const int64_t slot = a.k % h->sched->period();
   StepParams p{};
   fill_params(h, a, c0, c1, update_w, &p);
-  const bool has_m = a.momentum != 0.0f, has_ring = h->tau > 0;
-  const int arrays = 2 + (has_m ? 1 : 0) + (has_ring ? 1 : 0);
+  const bool has_m = a.M != nullptr, has_v = a.V != nullptr, has_ring = h->tau > 0;
+  const int arrays = 2 + (has_m ? 1 : 0) + (has_v ? 1 : 0) + (has_ring ? 1 : 0);
   int64_t tv = int64_t{1} << floor_log2(std::max<int64_t>(1, (pl.tile_cols > 0 ? pl.tile_cols : 256) / 4));
   tv = std::max<int64_t>(tv, 8);
   int stages = std::max(1, pl.stages);
@@ -319,7 +350,7 @@ int launch_tma(sgp_handle *h, const StepArgs &a, const Plan &pl, int64_t c0, int
   const int64_t tile_cols = tv * 4;
   const int64_t ntiles = (c1 - c0 + tile_cols - 1) / tile_cols;
   const int64_t grid = std::min<int64_t>(ntiles, static_cast<int64_t>(h->sm_count) * cps);
-  TmaKernel kern = pick_tma(has_m, a.nesterov != 0, a.Z != nullptr, has_ring);
+  TmaKernel kern = pick_tma(a.upd, a.Z != nullptr, has_ring);
   if (smem > 48 * 1024)
     SGP_CUDA_TRY(h, cudaFuncSetAttribute(reinterpret_cast<const void *>(kern),
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
@@ -332,18 +363,24 @@ int launch_tma(sgp_handle *h, const StepArgs &a, const Plan &pl, int64_t c0, int
   if (use_maps) use_maps = get_tensor_map(h, a.X, static_cast<int>(tile_cols), &maps.x);
   if (use_maps) use_maps = get_tensor_map(h, a.G, static_cast<int>(tile_cols), &maps.g);
   if (use_maps && has_m) use_maps = get_tensor_map(h, a.M, static_cast<int>(tile_cols), &maps.m);
+  if (use_maps && has_v) use_maps = get_tensor_map(h, a.V, static_cast<int>(tile_cols), &maps.v);
   if (use_maps && has_ring) use_maps = get_tensor_map(h, p.ring_x, static_cast<int>(tile_cols), &maps.r);
   kern<<<static_cast<unsigned>(grid), sgp::kTmaThreads, smem, stream>>>(p, ct, maps, stages, use_maps ? 1 : 0);
   SGP_CUDA_TRY(h, cudaGetLastError());
+  h->last_variant = use_maps ? 2 : 3;
+  h->last_grid = grid;
+  h->last_smem = static_cast<int64_t>(smem);
+  h->last_tile_cols = tile_cols;
   return SGP_OK;
 }
 
 // The whole step over columns [c0, c1): 128-bit kernel on the aligned bulk, scalar kernel on what is left.
 int launch_step_range(sgp_handle *h, const StepArgs &a, int64_t c0, int64_t c1, bool update_w, cudaStream_t stream) {
   const bool vec_ok = aligned16(a.X) && aligned16(a.G) && (a.M == nullptr || aligned16(a.M)) &&
-                      (a.Z == nullptr || aligned16(a.Z)) && (h->ld % 4 == 0) && (c0 % 4 == 0);
+                      (a.V == nullptr || aligned16(a.V)) && (a.Z == nullptr || aligned16(a.Z)) && (h->ld % 4 == 0) &&
+                      (c0 % 4 == 0);
   const int64_t vec_end = vec_ok ? c0 + ((c1 - c0) & ~int64_t{3}) : c0;
-  const int arrays = 2 + (a.M != nullptr ? 1 : 0) + (h->tau > 0 ? 1 : 0);
+  const int arrays = 2 + (a.M != nullptr ? 1 : 0) + (a.V != nullptr ? 1 : 0) + (h->tau > 0 ? 1 : 0);
   const int nnz = static_cast<int>(h->sched->slot(a.k).col.size());
   if (vec_end > c0) {
     const Plan pl = make_plan(h, arrays, a.M != nullptr, nnz, true);
@@ -492,7 +529,26 @@ int sgp_step(sgp_handle *h, float *d_X, float *d_W, float *d_M, const float *d_G
              float momentum, float weight_decay, int nesterov, void *stream) {
   const int rc = validate_step(h, d_X, d_W, d_M, d_G, k, momentum);
   if (rc != SGP_OK) return rc;
-  const StepArgs a{d_X, d_W, momentum != 0.0f ? d_M : nullptr, d_G, d_Z, k, lr, momentum, weight_decay, nesterov};
+  const StepArgs a{d_X, d_W, momentum != 0.0f ? d_M : nullptr, d_G, d_Z, k, lr, momentum, weight_decay,
+                   update_kind(momentum, nesterov)};
+  return launch_step_range(h, a, 0, h->d, true, static_cast<cudaStream_t>(stream));
+}
+
+int sgp_step_adam(sgp_handle *h, float *d_X, float *d_W, float *d_M1, float *d_M2, const float *d_G, float *d_Z,
+                  int64_t k, int64_t t, float lr, float beta1, float beta2, float eps, float weight_decay, void *stream) {
+  if (h == nullptr || d_X == nullptr || d_W == nullptr || d_M1 == nullptr || d_M2 == nullptr || d_G == nullptr ||
+      k < 0 || t < 1 || !(beta1 >= 0.0f && beta1 < 1.0f) || !(beta2 >= 0.0f && beta2 < 1.0f) || !(eps >= 0.0f))
+    return SGP_ERR_ARG;
+  StepArgs a{d_X, d_W, d_M1, d_G, d_Z, k, lr, 0.0f, weight_decay, sgp::kUpdAdam};
+  a.V = d_M2;
+  a.beta1 = beta1;
+  a.beta2 = beta2;
+  a.eps = eps;
+  // bias corrections in double, rounded once (t >= 1)
+  const double bc1 = 1.0 - std::pow(static_cast<double>(beta1), static_cast<double>(t));
+  const double bc2 = 1.0 - std::pow(static_cast<double>(beta2), static_cast<double>(t));
+  a.adam_step = static_cast<float>(static_cast<double>(lr) / bc1);
+  a.adam_rsqrt_bc2 = static_cast<float>(1.0 / std::sqrt(bc2));
   return launch_step_range(h, a, 0, h->d, true, static_cast<cudaStream_t>(stream));
 }
 
@@ -535,7 +591,7 @@ int sgp_step_host(sgp_handle *h, float *d_X, float *d_W, float *d_M, const float
   // earlier work of the caller on the legacy/default stream must be visible
   SGP_CUDA_TRY(h, cudaDeviceSynchronize());
   const StepArgs a{d_X, d_W, momentum != 0.0f ? d_M : nullptr, d_G, h_Z != nullptr ? d_Z : nullptr,
-                   k, lr, momentum, weight_decay, nesterov};
+                   k, lr, momentum, weight_decay, update_kind(momentum, nesterov)};
   const size_t pitch = static_cast<size_t>(h->ld) * sizeof(float);
   for (int64_t c = 0; c < nchunks; ++c) {
     const int64_t c0 = c * chunk_cols, c1 = std::min(h->d, c0 + chunk_cols);
@@ -637,6 +693,10 @@ int sgp_get_option(const sgp_handle *h, const char *key, int64_t *value) {
   else if (std::strcmp(key, "tile_cols") == 0) *value = h->opt_tile_cols;
   else if (std::strcmp(key, "ctas_per_sm") == 0) *value = h->opt_ctas_per_sm;
   else if (std::strcmp(key, "stages") == 0) *value = h->opt_stages;
+  else if (std::strcmp(key, "last_variant") == 0) *value = h->last_variant;
+  else if (std::strcmp(key, "last_grid") == 0) *value = h->last_grid;
+  else if (std::strcmp(key, "last_smem") == 0) *value = h->last_smem;
+  else if (std::strcmp(key, "last_tile_cols") == 0) *value = h->last_tile_cols;
   else return SGP_ERR_ARG;
   return SGP_OK;
 }

@@ -70,12 +70,12 @@ using StepKernel = void (*)(const sgp::StepParams, const sgp::ConstTable);
 
 template <int VEC>
 StepKernel pick(bool has_m, bool nesterov, bool has_z) {
-  if (!has_m) return has_z ? sgp::sgp_step_regs_kernel<VEC, false, false, true, false>
-                           : sgp::sgp_step_regs_kernel<VEC, false, false, false, false>;
-  if (nesterov) return has_z ? sgp::sgp_step_regs_kernel<VEC, true, true, true, false>
-                             : sgp::sgp_step_regs_kernel<VEC, true, true, false, false>;
-  return has_z ? sgp::sgp_step_regs_kernel<VEC, true, false, true, false>
-               : sgp::sgp_step_regs_kernel<VEC, true, false, false, false>;
+  if (!has_m) return has_z ? sgp::sgp_step_regs_kernel<VEC, sgp::kUpdSgd, true, false>
+                           : sgp::sgp_step_regs_kernel<VEC, sgp::kUpdSgd, false, false>;
+  if (nesterov) return has_z ? sgp::sgp_step_regs_kernel<VEC, sgp::kUpdNesterov, true, false>
+                             : sgp::sgp_step_regs_kernel<VEC, sgp::kUpdNesterov, false, false>;
+  return has_z ? sgp::sgp_step_regs_kernel<VEC, sgp::kUpdHeavyBall, true, false>
+               : sgp::sgp_step_regs_kernel<VEC, sgp::kUpdHeavyBall, false, false>;
 }
 
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }

@@ -13,7 +13,6 @@
 namespace sgp {
 
 constexpr int kThreads = 256;       // threads per CTA of the register-staged kernel
-constexpr int kItemsPerThread = 4;  // (row, vector-column) items a thread keeps in flight per batch
 
 // Mixing table of one step small enough to travel as a kernel argument (constant bank).
 constexpr int kConstRows = 64;
@@ -27,7 +26,8 @@ struct ConstTable {
 struct StepParams {
   float *X;
   float *W;
-  float *M;        // may be null when momentum == 0
+  float *M;        // momentum buffer / Adam first moment; null for plain SGD
+  float *V;        // Adam second moment; null otherwise
   const float *G;
   float *Z;        // may be null
   float *ring_x;   // this step's ring slot (n x ld) or null when tau == 0
@@ -40,7 +40,10 @@ struct StepParams {
   int log2_tile_vecs;  // tile width in vectors (power of two)
   int update_w;        // 1: this launch also commits W (and the weight ring) for the step
   int table_mode;      // 0: copy table from the kernel argument, 1: copy from global, 2: read global in place
+  int single_buffer;   // register kernel: 1 = one exchange tile and two barriers per tile (large n)
   float lr, momentum, wd;
+  // Adam only: decay rates, epsilon, lr / (1 - beta1^t) and 1 / sqrt(1 - beta2^t)
+  float beta1, beta2, eps, adam_step, adam_rsqrt_bc2;
   const int32_t *rowptr;  // global copy of the step's CSR (always valid)
   const int32_t *col;
   const float *val;
@@ -69,19 +72,43 @@ template <typename V> __device__ __forceinline__ V vzero();
 template <> __device__ __forceinline__ float4 vzero<float4>() { return make_float4(0.f, 0.f, 0.f, 0.f); }
 template <> __device__ __forceinline__ float vzero<float>() { return 0.f; }
 
-// Local update of one element group: returns h = x^(k+1/2) and the new momentum (Alg. 3 lines 4-5;
-// Alg. 1 line 4 when there is no momentum).  Weight decay adds wd * x to the gradient.
-template <bool HAS_M, bool NESTEROV, typename V>
-__device__ __forceinline__ V local_update(V x, V g, V &u, float lr, float momentum, float wd) {
-  V gt = vfma(wd, x, g);
-  V s;
-  if (HAS_M) {
-    u = vfma(momentum, u, gt);
-    s = NESTEROV ? vfma(momentum, u, gt) : u;
-  } else {
-    s = gt;
+__device__ __forceinline__ float4 vmulv(float4 a, float4 b) { return make_float4(a.x * b.x, a.y * b.y, a.z * b.z, a.w * b.w); }
+__device__ __forceinline__ float vmulv(float a, float b) { return a * b; }
+// a / (sqrt(v) * r + eps), IEEE square root and division
+__device__ __forceinline__ float adam_ratio(float a, float v, float r, float eps) { return a / fmaf(sqrtf(v), r, eps); }
+__device__ __forceinline__ float4 adam_ratio(float4 a, float4 v, float r, float eps) {
+  return make_float4(adam_ratio(a.x, v.x, r, eps), adam_ratio(a.y, v.y, r, eps), adam_ratio(a.z, v.z, r, eps),
+                     adam_ratio(a.w, v.w, r, eps));
+}
+
+// Which local optimiser runs on the biased numerators before the mix.
+enum : int { kUpdSgd = 0, kUpdHeavyBall = 1, kUpdNesterov = 2, kUpdAdam = 3 };
+template <int UPD> struct UpdTraits {
+  static constexpr bool kHasM = UPD != kUpdSgd;
+  static constexpr bool kHasV = UPD == kUpdAdam;
+  static constexpr int kItems = UPD == kUpdAdam ? 3 : 4;   // items a thread of the register kernel keeps in flight
+};
+
+// Local update of one element group: returns h = x^(k+1/2) and updates the optimiser state in place.
+// SGD: Alg. 1 line 4.  Momentum / Nesterov: Alg. 3 lines 4-5.  Adam (Sec. 6.2, App. C.1: "combine SGP
+// with the Adam preconditioner"): bias-corrected Adam step on the numerator, moments stay local.
+// Weight decay adds wd * x to the gradient in every case.
+template <int UPD, typename V>
+__device__ __forceinline__ V local_update(V x, V g, V &u, V &v, const StepParams &p) {
+  const V gt = vfma(p.wd, x, g);
+  if (UPD == kUpdAdam) {
+    u = vfma(p.beta1, u, vmul(1.0f - p.beta1, gt));
+    v = vfma(p.beta2, v, vmul(1.0f - p.beta2, vmulv(gt, gt)));
+    return vfma(-p.adam_step, adam_ratio(u, v, p.adam_rsqrt_bc2, p.eps), x);
   }
-  return vfma(-lr, s, x);
+  V s;
+  if (UPD == kUpdSgd) {
+    s = gt;
+  } else {
+    u = vfma(p.momentum, u, gt);
+    s = UPD == kUpdNesterov ? vfma(p.momentum, u, gt) : u;
+  }
+  return vfma(-p.lr, s, x);
 }
 
 // Shared-memory carve-up (dynamic): [H tile: tile_items vectors][w_old n][rw_in n][inv_w n][p_self n]
@@ -164,24 +191,26 @@ __device__ __forceinline__ CtaTables cta_prologue(const StepParams &p, const Con
 // writes x^(k+1/2) into a shared tile, one barrier, then gathers its receivers' rows from the tile.
 // The tile is double-buffered so one barrier per batch suffices.
 // ------------------------------------------------------------------------------------------------
-template <int VEC, bool HAS_M, bool NESTEROV, bool HAS_Z, bool HAS_RING>
+template <int VEC, int UPD, bool HAS_Z, bool HAS_RING>
 __global__ void __launch_bounds__(kThreads, 2)
 sgp_step_regs_kernel(const __grid_constant__ StepParams p, const __grid_constant__ ConstTable ct) {
   using V = typename VecT<VEC>::type;
+  constexpr bool HAS_M = UpdTraits<UPD>::kHasM;
+  constexpr bool HAS_V = UpdTraits<UPD>::kHasV;
+  constexpr int kItemsPerThread = UpdTraits<UPD>::kItems;
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int n = p.n;
   const int tv = 1 << p.log2_tile_vecs;
   const int tile_items = n * tv;
   V *H0 = reinterpret_cast<V *>(smem_raw);
-  V *H1 = H0 + tile_items;
-  float *scratch = reinterpret_cast<float *>(H1 + tile_items);
+  V *H1 = p.single_buffer ? H0 : H0 + tile_items;
+  float *scratch = reinterpret_cast<float *>(H0 + (p.single_buffer ? 1 : 2) * tile_items);
   const CtaTables tab = cta_prologue<HAS_RING>(p, ct, scratch, kThreads);
 
   const int64_t ld = p.ld;
   const int64_t ncols = p.col_end - p.col_begin;
   const int64_t tile_cols = static_cast<int64_t>(tv) * VEC;
   const int64_t ntiles = (ncols + tile_cols - 1) / tile_cols;
-  const float lr = p.lr, momentum = p.momentum, wd = p.wd;
   int buf = 0;
 
   for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
@@ -189,7 +218,7 @@ sgp_step_regs_kernel(const __grid_constant__ StepParams p, const __grid_constant
     V *H = buf ? H1 : H0;
     // ---- phase 1: local update, all batches of this tile
     for (int base = 0; base < tile_items; base += kThreads * kItemsPerThread) {
-      V x[kItemsPerThread], g[kItemsPerThread], u[kItemsPerThread];
+      V x[kItemsPerThread], g[kItemsPerThread], u[kItemsPerThread], vv[kItemsPerThread];
       bool ok[kItemsPerThread];
       int64_t off[kItemsPerThread];
 #pragma unroll
@@ -207,14 +236,16 @@ sgp_step_regs_kernel(const __grid_constant__ StepParams p, const __grid_constant
           x[q] = ld_stream(reinterpret_cast<const V *>(p.X + off[q]));
           g[q] = ld_stream(reinterpret_cast<const V *>(p.G + off[q]));
           if (HAS_M) u[q] = ld_stream(reinterpret_cast<const V *>(p.M + off[q]));
+          if (HAS_V) vv[q] = ld_stream(reinterpret_cast<const V *>(p.V + off[q]));
         }
       }
 #pragma unroll
       for (int q = 0; q < kItemsPerThread; ++q) {
         const int item = base + q * kThreads + threadIdx.x;
         if (ok[q]) {
-          const V h = local_update<HAS_M, NESTEROV, V>(x[q], g[q], u[q], lr, momentum, wd);
+          const V h = local_update<UPD, V>(x[q], g[q], u[q], vv[q], p);
           if (HAS_M) st_stream(reinterpret_cast<V *>(p.M + off[q]), u[q]);
+          if (HAS_V) st_stream(reinterpret_cast<V *>(p.V + off[q]), vv[q]);
           H[item] = h;
         } else if (item < tile_items) {
           H[item] = vzero<V>();
@@ -263,6 +294,7 @@ sgp_step_regs_kernel(const __grid_constant__ StepParams p, const __grid_constant
       }
     }
     buf ^= 1;
+    if (p.single_buffer) __syncthreads();   // the only tile is about to be overwritten
   }
 }
 
@@ -338,7 +370,7 @@ __device__ __forceinline__ void tma_load_2d(void *dst_smem, const CUtensorMap *m
 }
 // Tensor maps of the arrays a launch streams in (only those the launch uses are encoded).
 struct alignas(64) TmaMaps {
-  CUtensorMap x, g, m, r;
+  CUtensorMap x, g, m, v, r;
 };
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void consumer_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kTmaConsumers) : "memory"); }
@@ -356,12 +388,16 @@ __device__ __forceinline__ bool consumer_all(bool flag) {
   return out != 0;
 }
 
-template <bool HAS_M, bool NESTEROV, bool HAS_Z, bool HAS_RING>
+template <int UPD, bool HAS_Z, bool HAS_RING>
 __global__ void __launch_bounds__(kTmaThreads, 2)
 sgp_step_tma_kernel(const __grid_constant__ StepParams p, const __grid_constant__ ConstTable ct,
                     const __grid_constant__ TmaMaps maps, const int stages, const int use_tensor_maps) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
-  constexpr int kArrays = 2 + (HAS_M ? 1 : 0) + (HAS_RING ? 1 : 0);
+  constexpr bool HAS_M = UpdTraits<UPD>::kHasM;
+  constexpr bool HAS_V = UpdTraits<UPD>::kHasV;
+  // stage layout: [X][G][M if any][V if any][ring if any], each n x tile columns
+  constexpr int kIdxM = 2, kIdxV = 2 + (HAS_M ? 1 : 0), kIdxR = kIdxV + (HAS_V ? 1 : 0);
+  constexpr int kArrays = kIdxR + (HAS_RING ? 1 : 0);
   constexpr int kMaxStages = 8;
   const int n = p.n;
   const int tv = 1 << p.log2_tile_vecs;
@@ -414,9 +450,9 @@ sgp_step_tma_kernel(const __grid_constant__ StepParams p, const __grid_constant_
           mbar_arrive_expect_tx(full_bar + s, static_cast<uint32_t>(stage_bytes));
           tma_load_2d(stage, &maps.x, static_cast<int>(col0), 0, full_bar + s);
           tma_load_2d(stage + arr_bytes, &maps.g, static_cast<int>(col0), 0, full_bar + s);
-          if (HAS_M) tma_load_2d(stage + 2 * arr_bytes, &maps.m, static_cast<int>(col0), 0, full_bar + s);
-          if (HAS_RING)
-            tma_load_2d(stage + (2 + (HAS_M ? 1 : 0)) * arr_bytes, &maps.r, static_cast<int>(col0), 0, full_bar + s);
+          if (HAS_M) tma_load_2d(stage + kIdxM * arr_bytes, &maps.m, static_cast<int>(col0), 0, full_bar + s);
+          if (HAS_V) tma_load_2d(stage + kIdxV * arr_bytes, &maps.v, static_cast<int>(col0), 0, full_bar + s);
+          if (HAS_RING) tma_load_2d(stage + kIdxR * arr_bytes, &maps.r, static_cast<int>(col0), 0, full_bar + s);
         }
         issued = it + 1;
         continue;
@@ -428,7 +464,8 @@ sgp_step_tma_kernel(const __grid_constant__ StepParams p, const __grid_constant_
         const float *src;
         if (arr == 0) src = p.X;
         else if (arr == 1) src = p.G;
-        else if (arr == 2 && HAS_M) src = p.M;
+        else if (HAS_M && arr == kIdxM) src = p.M;
+        else if (HAS_V && arr == kIdxV) src = p.V;
         else src = p.ring_x;
         bulk_copy_g2s(stage + (static_cast<size_t>(arr) * tile_items + static_cast<size_t>(row) * tv) * sizeof(float4),
                       src + static_cast<int64_t>(row) * ld + col0, seg_bytes, full_bar + s);
@@ -445,7 +482,6 @@ sgp_step_tma_kernel(const __grid_constant__ StepParams p, const __grid_constant_
     }
   } else {
     // ---------------- consumer warps
-    const float lr = p.lr, momentum = p.momentum, wd = p.wd;
     const int ctid = threadIdx.x;
     for (int64_t it = 0; it < my_tiles; ++it) {
       const int s = static_cast<int>(it % stages);
@@ -461,8 +497,9 @@ sgp_step_tma_kernel(const __grid_constant__ StepParams p, const __grid_constant_
       const int64_t col0 = p.col_begin + tile * tile_cols;
       float4 *Xs = reinterpret_cast<float4 *>(smem_raw + s * stage_bytes);
       const float4 *Gs = Xs + tile_items;
-      const float4 *Ms = Gs + tile_items;
-      const float4 *Rs = Xs + static_cast<size_t>(2 + (HAS_M ? 1 : 0)) * tile_items;
+      const float4 *Ms = Xs + static_cast<size_t>(kIdxM) * tile_items;
+      const float4 *Vs = Xs + static_cast<size_t>(kIdxV) * tile_items;
+      const float4 *Rs = Xs + static_cast<size_t>(kIdxR) * tile_items;
       // phase 1: local update; x^(k+1/2) replaces x in the stage
       for (int item = ctid; item < tile_items; item += kTmaConsumers) {
         const int row = item >> p.log2_tile_vecs;
@@ -470,8 +507,10 @@ sgp_step_tma_kernel(const __grid_constant__ StepParams p, const __grid_constant_
         const int64_t col = col0 + static_cast<int64_t>(c) * 4;
         if (col < p.col_end) {
           float4 u = HAS_M ? Ms[item] : make_float4(0.f, 0.f, 0.f, 0.f);
-          const float4 h = local_update<HAS_M, NESTEROV, float4>(Xs[item], Gs[item], u, lr, momentum, wd);
+          float4 v2 = HAS_V ? Vs[item] : make_float4(0.f, 0.f, 0.f, 0.f);
+          const float4 h = local_update<UPD, float4>(Xs[item], Gs[item], u, v2, p);
           if (HAS_M) st_stream(reinterpret_cast<float4 *>(p.M + static_cast<int64_t>(row) * ld + col), u);
+          if (HAS_V) st_stream(reinterpret_cast<float4 *>(p.V + static_cast<int64_t>(row) * ld + col), v2);
           Xs[item] = h;
         }
       }

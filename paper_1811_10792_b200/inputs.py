@@ -107,6 +107,10 @@ class Workload:
     x0_shared: bool = False   # identical initial row on every node
     grad_std: float = 0.1
     seed: int = 181110792
+    optimizer: str = "sgd"          # "sgd" (plain / momentum / Nesterov by `momentum`, `nesterov`) or "adam"
+    beta1: float = 0.9
+    beta2: float = 0.98
+    adam_eps: float = 1e-8
 
     def scaled(self, d: int, K: int | None = None) -> "Workload":
         """Same recipe on a shorter parameter vector (parity tests, CPU baseline samples)."""
@@ -128,6 +132,11 @@ WORKLOADS = {
     "resnet50_osgp1": Workload("resnet50_osgp1", n=32, d=25_557_032, K=20, graph="exp", peers=1, lr=0.1,
                                momentum=0.9, tau=1, x0_std=0.1, x0_shared=True, grad_std=0.1, seed=181110796),
 }
+
+# Adam-SGP on the Transformer-sized vector (the paper's translation runs combine SGP with Adam)
+WORKLOADS["transformer_adam"] = Workload("transformer_adam", n=16, d=61_000_000, K=20, graph="exp", peers=2, lr=1e-3,
+                                         x0_std=math.sqrt(0.02), grad_std=math.sqrt(1e-3), seed=181110798,
+                                         optimizer="adam")
 
 SWEEP_N = (4, 16, 64, 256)
 SWEEP_D = (10_000, 1_000_000, 10_000_000, 100_000_000)
