@@ -178,6 +178,16 @@ int sgp_ring_import(sgp_handle *h, const float *d_ring_x, const float *d_ring_w,
 int sgp_check(sgp_handle *h, const float *d_X, const float *d_W, double *h_stats, void *stream);
 
 /*
+ * sgp_param_deviation: the parameter-deviation diagnostic of Sec. 6.1 / Fig. 2.  For an n x ld device
+ * array A (X, Z or any other per-node array of this handle's shape) writes to HOST h_dev[n] the
+ * Euclidean distance of every node's row from the node-wise average row,
+ *     h_dev[i] = || A_i - (1/n) sum_j A_j ||_2 ;
+ * the figure plots the mean with the min..max band of these n numbers.  One read of A (4 bytes per
+ * element); squared differences are accumulated in fp32 per CTA and in fp64 across CTAs.  Synchronises.
+ */
+int sgp_param_deviation(sgp_handle *h, const float *d_A, double *h_dev, void *stream);
+
+/*
  * Tuning knobs for experiments (defaults are chosen per problem shape):
  *   "variant"      0 = automatic, 1 = register-staged kernel, 2 = TMA pipelined kernel fed by 2-D tensor
  *                  maps, 3 = the same kernel fed by one bulk copy per row segment (no tensor maps)

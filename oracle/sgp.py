@@ -167,3 +167,9 @@ def total_mass(st: SGPState):
         sx = sx + mx.sum(axis=0)
         sw = sw + mw.sum()
     return sx, sw
+
+
+def param_deviation(a):
+    """Sec. 6.1 "Parameter deviations": distance of every node's row from the node-wise average row."""
+    a = np.asarray(a, dtype=np.float64)
+    return np.linalg.norm(a - a.mean(axis=0, keepdims=True), axis=1)

@@ -92,4 +92,44 @@ __global__ void __launch_bounds__(256) sgp_weight_scan_kernel(const float *__res
   }
 }
 
+// Parameter deviation (Sec. 6.1 "Parameter deviations", Fig. 2): out[i] += sum over this CTA's columns of
+// (A[i][c] - mean_j A[j][c])^2.  A CTA stages n rows x tile_cols columns in shared memory, forms the
+// column means, then every warp reduces whole rows.  One read of A, nothing else.
+__global__ void __launch_bounds__(256) sgp_deviation_kernel(const float *__restrict__ A, int n, int64_t d, int64_t ld,
+                                                             int tile_cols, double *out) {
+  extern __shared__ float dev_smem[];
+  float *tile = dev_smem;                         // n x tile_cols
+  float *mean = tile + static_cast<size_t>(n) * tile_cols;
+  float *acc = mean + tile_cols;                  // n partial sums of this CTA
+  for (int i = threadIdx.x; i < n; i += blockDim.x) acc[i] = 0.f;
+  const int64_t ntiles = (d + tile_cols - 1) / tile_cols;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+  const float inv_n = 1.0f / static_cast<float>(n);
+  for (int64_t t = blockIdx.x; t < ntiles; t += gridDim.x) {
+    const int64_t col0 = t * tile_cols;
+    const int valid = static_cast<int>(min(static_cast<int64_t>(tile_cols), d - col0));
+    __syncthreads();
+    for (int r = warp; r < n; r += nwarps)
+      for (int c = lane; c < valid; c += 32) tile[r * tile_cols + c] = __ldcs(A + static_cast<int64_t>(r) * ld + col0 + c);
+    __syncthreads();
+    for (int c = threadIdx.x; c < valid; c += blockDim.x) {
+      float s = 0.f;
+      for (int r = 0; r < n; ++r) s += tile[r * tile_cols + c];
+      mean[c] = s * inv_n;
+    }
+    __syncthreads();
+    for (int r = warp; r < n; r += nwarps) {
+      float q = 0.f;
+      for (int c = lane; c < valid; c += 32) {
+        const float e = tile[r * tile_cols + c] - mean[c];
+        q = fmaf(e, e, q);
+      }
+      for (int o = 16; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
+      if (lane == 0) acc[r] += q;                 // row r belongs to this warp only: no race
+    }
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < n; i += blockDim.x) atomicAdd(out + i, static_cast<double>(acc[i]));
+}
+
 }  // namespace sgp

@@ -35,7 +35,7 @@ struct sgp_handle {
   float *ring_x = nullptr;   // tau * n * ld
   float *ring_w = nullptr;   // tau * n
   unsigned *d_words = nullptr;  // [0] ticket, [1] status
-  double *d_stats = nullptr;    // 4 doubles for sgp_check
+  double *d_stats = nullptr;    // 4 doubles for sgp_check, then SGP_MAX_NODES doubles for sgp_param_deviation
   int64_t opt_variant = 0, opt_tile_cols = 0, opt_ctas_per_sm = 0, opt_stages = 0;
   int64_t last_variant = 0, last_grid = 0, last_smem = 0, last_tile_cols = 0;   // of the most recent step launch
   cudaStream_t s_h2d = nullptr, s_compute = nullptr, s_d2h = nullptr;
@@ -486,7 +486,7 @@ int sgp_create(sgp_handle **out, int n, int64_t d, int64_t ld, const sgp_graph_d
   if (e != cudaSuccess) return fail(SGP_ERR_ALLOC, e);
   e = cudaMalloc(&h->d_words, 2 * sizeof(unsigned));
   if (e != cudaSuccess) return fail(SGP_ERR_ALLOC, e);
-  e = cudaMalloc(&h->d_stats, 4 * sizeof(double));
+  e = cudaMalloc(&h->d_stats, (4 + SGP_MAX_NODES) * sizeof(double));
   if (e != cudaSuccess) return fail(SGP_ERR_ALLOC, e);
   if (tau > 0) {
     e = cudaMalloc(&h->ring_x, static_cast<size_t>(tau) * n * ld * sizeof(float));
@@ -664,6 +664,28 @@ int sgp_check(sgp_handle *h, const float *d_X, const float *d_W, double *h_stats
   h_stats[1] = tmp[3];
   h_stats[2] = tmp[1];
   h_stats[3] = tmp[0];
+  return SGP_OK;
+}
+
+int sgp_param_deviation(sgp_handle *h, const float *d_A, double *h_dev, void *stream) {
+  if (h == nullptr || d_A == nullptr || h_dev == nullptr) return SGP_ERR_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  double *acc = h->d_stats + 4;
+  SGP_CUDA_TRY(h, cudaMemsetAsync(acc, 0, static_cast<size_t>(h->n) * sizeof(double), st));
+  // tile of n rows x tile_cols columns in shared memory, at most ~64 KB
+  int tile_cols = 256;
+  while (tile_cols > 32 && static_cast<size_t>(h->n) * tile_cols * 4 > 64 * 1024) tile_cols >>= 1;
+  const size_t smem = (static_cast<size_t>(h->n) * tile_cols + tile_cols + h->n) * sizeof(float);
+  if (smem > 48 * 1024)
+    SGP_CUDA_TRY(h, cudaFuncSetAttribute(reinterpret_cast<const void *>(sgp::sgp_deviation_kernel),
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  const int64_t ntiles = (h->d + tile_cols - 1) / tile_cols;
+  const unsigned grid = static_cast<unsigned>(std::min<int64_t>(ntiles, static_cast<int64_t>(h->sm_count) * 2));
+  sgp::sgp_deviation_kernel<<<grid, 256, smem, st>>>(d_A, h->n, h->d, h->ld, tile_cols, acc);
+  SGP_CUDA_TRY(h, cudaGetLastError());
+  SGP_CUDA_TRY(h, cudaMemcpyAsync(h_dev, acc, static_cast<size_t>(h->n) * sizeof(double), cudaMemcpyDeviceToHost, st));
+  SGP_CUDA_TRY(h, cudaStreamSynchronize(st));
+  for (int i = 0; i < h->n; ++i) h_dev[i] = std::sqrt(h_dev[i]);
   return SGP_OK;
 }
 

@@ -301,3 +301,20 @@ def test_adam_sgp_moments_stay_local_and_mass_is_mixed():
     assert np.allclose(st.u, m, rtol=1e-13) and np.allclose(st.v, v, rtol=1e-13)     # independent of the graph
     _, sw = O.total_mass(st)
     assert abs(sw - n) < 1e-12
+
+
+# ---------------------------------------------------------------- parameter deviation (Fig. 2 metric)
+def test_param_deviation_closed_forms():
+    a = np.array([3.0, -4.0, 12.0])
+    # two nodes at +a and -a: the average is 0, each is ||a|| = 13 away
+    assert np.allclose(O.param_deviation(np.stack([a, -a])), [13.0, 13.0])
+    # a common shift changes nothing; consensus gives zero
+    rng = np.random.default_rng(60)
+    x = rng.standard_normal((6, 50))
+    assert np.allclose(O.param_deviation(x + 7.5), O.param_deviation(x), rtol=1e-12)
+    assert np.all(O.param_deviation(np.tile(x[0], (6, 1))) < 1e-14)
+    # one node displaced by e from n-1 identical ones: it is (n-1)/n*||e|| away, the others ||e||/n
+    e = rng.standard_normal(50)
+    y = np.tile(x[0], (6, 1)); y[2] += e
+    want = np.full(6, np.linalg.norm(e) / 6); want[2] *= 5
+    assert np.allclose(O.param_deviation(y), want, rtol=1e-12)

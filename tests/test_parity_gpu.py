@@ -364,3 +364,19 @@ def test_bulk_copy_kernel_with_row_pitch(binding, inputs):
     for variant in (2, 3):
         out = _run_gpu(binding, inputs, w, ld=w.d + 8, offset=4, options={"variant": variant})
         _compare(w, out)
+
+
+def test_param_deviation_matches_oracle(binding, inputs):
+    from oracle import sgp as osgp
+    for n, d, pitch in ((32, 10_007, 256), (5, 300, 1), (256, 1029, 1), (16, 65_536, 256)):
+        A, ld = binding.empty_matrix(n, d, device=DEV, pitch_multiple=pitch, fill=float("nan"))
+        inputs.fill_normal(A, seed=77, stream=1, step=0, std=0.5)
+        A += torch.linspace(-1, 1, n, device=DEV)[:, None]            # nodes really differ
+        with binding.Sgp(n, d, binding.GraphDesc.exp_peers(1), ld=ld) as h:
+            got = h.param_deviation(A)
+        want = osgp.param_deviation(A.cpu().numpy())
+        assert np.allclose(got, want, rtol=2e-6), (n, d, np.abs(got / want - 1).max())
+    A, ld = binding.empty_matrix(8, 1000, device=DEV)
+    A[:] = torch.randn(1000, device=DEV)
+    with binding.Sgp(8, 1000, binding.GraphDesc.exp_peers(1), ld=ld) as h:
+        assert np.all(h.param_deviation(A) <= 1e-5)                   # consensus: zero deviation
