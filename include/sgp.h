@@ -194,6 +194,8 @@ int sgp_param_deviation(sgp_handle *h, const float *d_A, double *h_dev, void *st
  *   "tile_cols"    columns per tile (multiple of 4; 0 = automatic)
  *   "ctas_per_sm"  persistent CTAs per SM (0 = automatic)
  *   "stages"       shared-memory stages of the bulk-copy pipeline (0 = automatic, at most 8)
+ *   "l2_hint"      L2 evict-first policy on the pipeline's bulk copies: 0 = automatic (gradients only),
+ *                  1 = every array, 2 = none, 3 = gradients only, 4 = every array but the gradients
  * Read-only through sgp_get_option: "last_variant", "last_grid", "last_smem", "last_tile_cols" describe
  * the most recent step launch of the handle (which kernel ran, CTAs, dynamic shared memory, tile width).
  * Unknown keys or unsupported values return SGP_ERR_ARG and change nothing.

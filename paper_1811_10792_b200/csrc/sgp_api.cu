@@ -36,7 +36,7 @@ struct sgp_handle {
   float *ring_w = nullptr;   // tau * n
   unsigned *d_words = nullptr;  // [0] ticket, [1] status
   double *d_stats = nullptr;    // 4 doubles for sgp_check, then SGP_MAX_NODES doubles for sgp_param_deviation
-  int64_t opt_variant = 0, opt_tile_cols = 0, opt_ctas_per_sm = 0, opt_stages = 0;
+  int64_t opt_variant = 0, opt_tile_cols = 0, opt_ctas_per_sm = 0, opt_stages = 0, opt_l2_hint = 0;
   int64_t last_variant = 0, last_grid = 0, last_smem = 0, last_tile_cols = 0;   // of the most recent step launch
   cudaStream_t s_h2d = nullptr, s_compute = nullptr, s_d2h = nullptr;
   std::vector<cudaEvent_t> ev_in, ev_done;
@@ -215,6 +215,19 @@ Plan make_plan(const sgp_handle *h, int arrays, bool has_m, int nnz, bool vec) {
       while (pl.tile_cols > 32 && copies * static_cast<size_t>(h->n) * pl.tile_cols * 4 + fixed > 80 * 1024) pl.tile_cols >>= 1;
     }
   }
+  if (h->opt_variant > 0 && (h->opt_variant == 1) != (pl.variant == 1)) {
+    // the caller forces the other kernel family: take that family's defaults
+    if (h->opt_variant == 1) {
+      pl = Plan{1, 256, 2, 0};
+      if (vec) {
+        pl.tile_cols = std::max<int64_t>(256, int64_t{4} << floor_log2(std::max<int64_t>(1, 2048 / h->n)));
+        const size_t copies = h->n > 128 ? 1 : 2;
+        while (pl.tile_cols > 32 && copies * static_cast<size_t>(h->n) * pl.tile_cols * 4 > 76 * 1024) pl.tile_cols >>= 1;
+      }
+    } else {
+      pl = Plan{static_cast<int>(h->opt_variant), 256, 2, 2};
+    }
+  }
   if (h->opt_variant > 0) pl.variant = static_cast<int>(h->opt_variant);
   if (h->opt_tile_cols > 0) pl.tile_cols = h->opt_tile_cols;
   if (h->opt_stages > 0) pl.stages = static_cast<int>(h->opt_stages);
@@ -350,6 +363,7 @@ int launch_tma(sgp_handle *h, const StepArgs &a, const Plan &pl, int64_t c0, int
   const int64_t tile_cols = tv * 4;
   const int64_t ntiles = (c1 - c0 + tile_cols - 1) / tile_cols;
   const int64_t grid = std::min<int64_t>(ntiles, static_cast<int64_t>(h->sm_count) * cps);
+  p.l2_hint = h->opt_l2_hint == 2 ? 0 : (h->opt_l2_hint == 0 ? 3 : static_cast<int>(h->opt_l2_hint));
   TmaKernel kern = pick_tma(a.upd, a.Z != nullptr, has_ring);
   if (smem > 48 * 1024)
     SGP_CUDA_TRY(h, cudaFuncSetAttribute(reinterpret_cast<const void *>(kern),
@@ -703,6 +717,9 @@ int sgp_set_option(sgp_handle *h, const char *key, int64_t value) {
   } else if (std::strcmp(key, "stages") == 0) {
     if (value > 8) return SGP_ERR_ARG;
     h->opt_stages = value;
+  } else if (std::strcmp(key, "l2_hint") == 0) {
+    if (value > 4) return SGP_ERR_ARG;
+    h->opt_l2_hint = value;
   } else {
     return SGP_ERR_ARG;
   }
@@ -715,6 +732,7 @@ int sgp_get_option(const sgp_handle *h, const char *key, int64_t *value) {
   else if (std::strcmp(key, "tile_cols") == 0) *value = h->opt_tile_cols;
   else if (std::strcmp(key, "ctas_per_sm") == 0) *value = h->opt_ctas_per_sm;
   else if (std::strcmp(key, "stages") == 0) *value = h->opt_stages;
+  else if (std::strcmp(key, "l2_hint") == 0) *value = h->opt_l2_hint;
   else if (std::strcmp(key, "last_variant") == 0) *value = h->last_variant;
   else if (std::strcmp(key, "last_grid") == 0) *value = h->last_grid;
   else if (std::strcmp(key, "last_smem") == 0) *value = h->last_smem;
