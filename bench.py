@@ -202,6 +202,50 @@ def workload_config(w, extra=None):
     return cfg
 
 
+def run_sweep(args):
+    """Scaling sweep (random digraphs, Nesterov, Z written): one JSON line per (n, d) point that fits 150 GB."""
+    import torch
+    from paper_1811_10792_b200 import binding, inputs
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    from parity_util import graph_desc
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peak, peak_kind = measured_peak()
+    for n in inputs.SWEEP_N:
+        for d in inputs.SWEEP_D:
+            if 4 * 4 * n * d > 150e9:
+                continue                                    # (256, 1e8): 410 GB for X, M, G, Z
+            w = inputs.sweep_workload(n, d)
+            X, ld = binding.empty_matrix(n, d, device=dev, pitch_multiple=args.ld_align)
+            X.copy_(inputs.initial_x(w, device=dev))
+            M, _ = binding.empty_matrix(n, d, device=dev, pitch_multiple=args.ld_align, fill=0.0)
+            Z, _ = binding.empty_matrix(n, d, device=dev, pitch_multiple=args.ld_align)
+            G, _ = binding.empty_matrix(n, d, device=dev, pitch_multiple=args.ld_align)
+            inputs.gradient(w, 0, G)
+            Wt = torch.ones(n, device=dev)
+            K = w.K
+            with binding.Sgp(n, d, graph_desc(w, binding), ld=ld) as h:
+                for k in range(max(3, args.warmup)):
+                    h.step(X, Wt, M, G, Z, k, w.lr, w.momentum, 0.0, True)
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for k in range(K):
+                    h.step(X, Wt, M, G, Z, 3 + k, w.lr, w.momentum, 0.0, True)
+                e1.record()
+                torch.cuda.synchronize()
+                ms = e0.elapsed_time(e1) / K
+                launch = {k: h.get_option(k) for k in ("last_variant", "last_grid", "last_tile_cols")}
+            achieved = 24.0 * n * d / (ms * 1e-3) / 1e9
+            print(json.dumps({"metric": METRIC, "value": n * d / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": K,
+                              "ms_per_step": ms, "dtype": "f32", "data": "synthetic",
+                              "config": workload_config(w, extra={"row_pitch_floats": ld, **launch}),
+                              "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                                           "frac": achieved / peak, "peak_kind": f"of {peak_kind}"}}), flush=True)
+            del X, M, Z, G
+            torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -216,8 +260,12 @@ def main():
     ap.add_argument("--option", action="append", default=[], help="key=value passed to sgp_set_option")
     ap.add_argument("--ld-align", type=int, default=256,
                     help="row pitch of every n x d array is rounded up to this many floats (256 = 1 KB rows)")
+    ap.add_argument("--sweep", action="store_true", help="run every scaling-sweep point, one JSON line each")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.sweep:
+        run_sweep(args)
+        return
 
     from paper_1811_10792_b200 import inputs
     if args.workload.startswith("sweep:"):            # sweep:<n>:<d>  (scaling-sweep point, random digraphs)

@@ -5,6 +5,8 @@
 #include <algorithm>
 #include <cmath>
 #include <cstring>
+#include <map>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -91,6 +93,35 @@ void free_handle(sgp_handle *h) {
 }
 
 using StepKernel = void (*)(const StepParams, const ConstTable);
+
+// Per-kernel facts that do not change during the process: registers, static shared memory, and the
+// largest dynamic shared-memory size already enabled (so the attribute calls leave the launch path).
+struct KernelInfo {
+  int num_regs = 0;
+  size_t static_smem = 0;
+  size_t enabled_smem = 48 * 1024;
+};
+std::mutex g_kernel_info_mutex;
+std::map<const void *, KernelInfo> g_kernel_info;
+
+int kernel_info(sgp_handle *h, const void *kern, size_t smem, KernelInfo *out) {
+  std::lock_guard<std::mutex> lock(g_kernel_info_mutex);
+  auto it = g_kernel_info.find(kern);
+  if (it == g_kernel_info.end()) {
+    cudaFuncAttributes fa;
+    SGP_CUDA_TRY(h, cudaFuncGetAttributes(&fa, kern));
+    KernelInfo ki;
+    ki.num_regs = fa.numRegs;
+    ki.static_smem = fa.sharedSizeBytes;
+    it = g_kernel_info.emplace(kern, ki).first;
+  }
+  if (smem > it->second.enabled_smem) {
+    SGP_CUDA_TRY(h, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+    it->second.enabled_smem = smem;
+  }
+  *out = it->second;
+  return SGP_OK;
+}
 
 template <int VEC, int UPD>
 StepKernel pick_regs_flags(bool has_z, bool has_ring) {
@@ -248,6 +279,9 @@ int launch_regs(sgp_handle *h, const StepArgs &a, const Plan &pl, int64_t c0, in
   int64_t tv = int64_t{1} << floor_log2(std::max<int64_t>(1, sgp::kThreads * 4 / h->n));
   if (pl.tile_cols > 0) tv = int64_t{1} << floor_log2(std::max<int64_t>(1, pl.tile_cols / vec));
   tv = std::max<int64_t>(tv, min_tv);
+  // short rows: narrower tiles until there is about a tile per SM (launch-latency regime)
+  if (h->opt_tile_cols == 0)
+    while (tv > min_tv && tv * vec > 128 && (ncols + tv * vec - 1) / (tv * vec) < h->sm_count) tv >>= 1;
   const size_t table_bytes = table_smem_bytes(h, p.nnz);
   if (h->const_ok[static_cast<size_t>(slot)]) p.table_mode = 0;
   else p.table_mode = table_bytes <= 40 * 1024 ? 1 : 2;
@@ -266,19 +300,19 @@ int launch_regs(sgp_handle *h, const StepArgs &a, const Plan &pl, int64_t c0, in
   const int64_t ntiles = (ncols + tile_cols - 1) / tile_cols;
   StepKernel kern = vec == 4 ? pick_regs<4>(a.upd, a.Z != nullptr, h->tau > 0)
                              : pick_regs<1>(a.upd, a.Z != nullptr, h->tau > 0);
-  if (smem > 48 * 1024)
-    SGP_CUDA_TRY(h, cudaFuncSetAttribute(reinterpret_cast<const void *>(kern),
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  KernelInfo ki;
+  {
+    const int rc = kernel_info(h, reinterpret_cast<const void *>(kern), smem, &ki);
+    if (rc != SGP_OK) return rc;
+  }
   int cps = pl.cps;
   if (cps <= 0) {
     // Persistent grid of exactly one wave: CTAs resident per SM by registers, shared memory and threads.
     // (Computed here rather than asked of the occupancy calculator, whose answer depends on the
     // shared-memory carve-out it assumes; the hardware picks the carve-out that fits the launch.)
-    cudaFuncAttributes fa;
-    SGP_CUDA_TRY(h, cudaFuncGetAttributes(&fa, reinterpret_cast<const void *>(kern)));
-    const int regs_per_cta = ((fa.numRegs + 7) / 8 * 8) * sgp::kThreads;
+    const int regs_per_cta = ((ki.num_regs + 7) / 8 * 8) * sgp::kThreads;
     const int by_regs = regs_per_cta > 0 ? 65536 / regs_per_cta : 8;
-    const int by_smem = static_cast<int>((227 * 1024) / (smem + fa.sharedSizeBytes + 1024));
+    const int by_smem = static_cast<int>((227 * 1024) / (smem + ki.static_smem + 1024));
     cps = std::max(1, std::min({by_regs, by_smem, 2048 / sgp::kThreads}));
   }
   const int64_t grid = std::min<int64_t>(ntiles, static_cast<int64_t>(h->sm_count) * cps);
@@ -365,9 +399,11 @@ int launch_tma(sgp_handle *h, const StepArgs &a, const Plan &pl, int64_t c0, int
   const int64_t grid = std::min<int64_t>(ntiles, static_cast<int64_t>(h->sm_count) * cps);
   p.l2_hint = h->opt_l2_hint == 2 ? 0 : (h->opt_l2_hint == 0 ? 3 : static_cast<int>(h->opt_l2_hint));
   TmaKernel kern = pick_tma(a.upd, a.Z != nullptr, has_ring);
-  if (smem > 48 * 1024)
-    SGP_CUDA_TRY(h, cudaFuncSetAttribute(reinterpret_cast<const void *>(kern),
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  {
+    KernelInfo ki;
+    const int rc = kernel_info(h, reinterpret_cast<const void *>(kern), smem, &ki);
+    if (rc != SGP_OK) return rc;
+  }
   static const ConstTable kEmptyTable{};
   const ConstTable &ct = p.table_mode == 0 ? h->const_tables[static_cast<size_t>(slot)] : kEmptyTable;
   // 2-D tensor maps (one copy per array per tile) when the box fits; else one bulk copy per row segment
@@ -397,7 +433,9 @@ int launch_step_range(sgp_handle *h, const StepArgs &a, int64_t c0, int64_t c1, 
   const int arrays = 2 + (a.M != nullptr ? 1 : 0) + (a.V != nullptr ? 1 : 0) + (h->tau > 0 ? 1 : 0);
   const int nnz = static_cast<int>(h->sched->slot(a.k).col.size());
   if (vec_end > c0) {
-    const Plan pl = make_plan(h, arrays, a.M != nullptr, nnz, true);
+    Plan pl = make_plan(h, arrays, a.M != nullptr, nnz, true);
+    // short rows (fewer 1 KB tiles than SMs): the register kernel with narrow tiles spreads them better
+    if (h->opt_variant == 0 && pl.variant >= 2 && (vec_end - c0) < int64_t{256} * h->sm_count) pl = Plan{1, 256, 2, 0};
     int rc = SGP_ERR_STATE;
     if (pl.variant >= 2) rc = launch_tma(h, a, pl, c0, vec_end, update_w && vec_end == c1, stream);
     if (rc == SGP_ERR_STATE) {

@@ -380,3 +380,40 @@ def test_param_deviation_matches_oracle(binding, inputs):
     A[:] = torch.randn(1000, device=DEV)
     with binding.Sgp(8, 1000, binding.GraphDesc.exp_peers(1), ld=ld) as h:
         assert np.all(h.param_deviation(A) <= 1e-5)                   # consensus: zero deviation
+
+
+@pytest.mark.parametrize("variant", [1, 3])
+def test_steps_can_be_captured_in_a_cuda_graph(binding, inputs, variant):
+    """One schedule period captured once and replayed: same bits as eager launches (launch-bound small cases)."""
+    w = inputs.sweep_workload(16, 10_000)
+    n, d = w.n, w.d
+    period = 10
+    def fresh():
+        return (inputs.initial_x(w, device=DEV).contiguous(), torch.ones(n, device=DEV), torch.zeros((n, d), device=DEV),
+                torch.empty((n, d), device=DEV))
+    G = [inputs.gradient(w, k, torch.empty((n, d), device=DEV)) for k in range(period)]
+    X, W, M, Z = fresh()
+    with binding.Sgp(n, d, graph_desc(w, binding)) as h:
+        h.set_option("variant", variant)
+        for rep in range(2):
+            for k in range(period):
+                h.step(X, W, M, G[k], Z, rep * period + k, w.lr, w.momentum, 0.0, True)
+        torch.cuda.synchronize()
+    X2, W2, M2, Z2 = fresh()
+    with binding.Sgp(n, d, graph_desc(w, binding)) as h:
+        h.set_option("variant", variant)
+        h.step(X2, W2, M2, G[0], Z2, 0, w.lr, w.momentum, 0.0, True)       # warm-up outside capture (sets attributes)
+        torch.cuda.synchronize()
+        X2, W2, M2, Z2 = fresh()
+        side = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                for k in range(period):
+                    h.step(X2, W2, M2, G[k], Z2, k, w.lr, w.momentum, 0.0, True, stream=side)
+        graph.replay()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert h.device_status() == 0
+    for a, b in ((X, X2), (W, W2), (M, M2), (Z, Z2)):
+        assert torch.equal(a, b)
