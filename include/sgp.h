@@ -194,6 +194,8 @@ int sgp_param_deviation(sgp_handle *h, const float *d_A, double *h_dev, void *st
  *   "tile_cols"    columns per tile (multiple of 4; 0 = automatic)
  *   "ctas_per_sm"  persistent CTAs per SM (0 = automatic)
  *   "stages"       shared-memory stages of the bulk-copy pipeline (0 = automatic, at most 8)
+ *   "single_buffer" register-staged kernel: 0 = automatic (n > 128), 1 = one exchange tile and two barriers
+ *                  per tile, 2 = two exchange tiles and one barrier
  *   "l2_hint"      L2 evict-first policy on the pipeline's bulk copies: 0 = automatic (gradients only),
  *                  1 = every array, 2 = none, 3 = gradients only, 4 = every array but the gradients
  * Read-only through sgp_get_option: "last_variant", "last_grid", "last_smem", "last_tile_cols" describe

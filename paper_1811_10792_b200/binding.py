@@ -177,7 +177,7 @@ class Schedule(_ScheduleView):
         super().__init__(ptr, n)
 
     def close(self):
-        if getattr(self, "_ptr", None):
+        if getattr(self, "_ptr", None) and _lib is not None:
             _lib.sgp_schedule_destroy(self._ptr)
             self._ptr = None
 
@@ -204,7 +204,7 @@ class Sgp:
         _check(_lib.sgp_create(C.byref(self._h), n, d, self.ld, C.byref(graph.c), tau, flags), "sgp_create")
 
     def close(self):
-        if getattr(self, "_h", None):
+        if getattr(self, "_h", None) and _lib is not None:      # _lib is None during interpreter shutdown
             _lib.sgp_destroy(self._h)
             self._h = None
 

@@ -38,7 +38,7 @@ struct sgp_handle {
   float *ring_w = nullptr;   // tau * n
   unsigned *d_words = nullptr;  // [0] ticket, [1] status
   double *d_stats = nullptr;    // 4 doubles for sgp_check, then SGP_MAX_NODES doubles for sgp_param_deviation
-  int64_t opt_variant = 0, opt_tile_cols = 0, opt_ctas_per_sm = 0, opt_stages = 0, opt_l2_hint = 0;
+  int64_t opt_variant = 0, opt_tile_cols = 0, opt_ctas_per_sm = 0, opt_stages = 0, opt_l2_hint = 0, opt_single_buffer = 0;
   int64_t last_variant = 0, last_grid = 0, last_smem = 0, last_tile_cols = 0;   // of the most recent step launch
   cudaStream_t s_h2d = nullptr, s_compute = nullptr, s_d2h = nullptr;
   std::vector<cudaEvent_t> ev_in, ev_done;
@@ -216,6 +216,11 @@ struct Plan {
   int cps;
 };
 
+// Register-staged kernel: one exchange tile (two barriers per tile) where that keeps the row segments at
+// 1 KB (32 < n <= 64: 0.95 against 0.92) or at 256 B (n > 128: 0.91 against 0.70); two tiles and one
+// barrier elsewhere (n = 128: 0.94 against 0.91).
+bool auto_single_buffer(int n) { return (n > 32 && n <= 64) || n > 128; }
+
 size_t table_smem_bytes(const sgp_handle *h, int nnz) { return (static_cast<size_t>(h->n) + 1 + 2 * static_cast<size_t>(nnz)) * 4; }
 
 // Heuristics from measurements on B200.  The step is HBM-bound; what decides the achieved bandwidth
@@ -242,7 +247,7 @@ Plan make_plan(const sgp_handle *h, int arrays, bool has_m, int nnz, bool vec) {
       pl.tile_cols = std::max<int64_t>(256, int64_t{4} << floor_log2(std::max<int64_t>(1, 2048 / h->n)));
       // keep the two resident CTAs' shared memory near half of the SM's 256 KB: the rest is the L1 that
       // tracks the loads in flight (measured: n = 48 at 2 x 100 KB reaches 0.74, at 2 x 50 KB 0.93)
-      const size_t copies = h->n > 128 ? 1 : 2;
+      const size_t copies = auto_single_buffer(h->n) ? 1 : 2;
       while (pl.tile_cols > 32 && copies * static_cast<size_t>(h->n) * pl.tile_cols * 4 + fixed > 80 * 1024) pl.tile_cols >>= 1;
     }
   }
@@ -252,7 +257,7 @@ Plan make_plan(const sgp_handle *h, int arrays, bool has_m, int nnz, bool vec) {
       pl = Plan{1, 256, 2, 0};
       if (vec) {
         pl.tile_cols = std::max<int64_t>(256, int64_t{4} << floor_log2(std::max<int64_t>(1, 2048 / h->n)));
-        const size_t copies = h->n > 128 ? 1 : 2;
+        const size_t copies = auto_single_buffer(h->n) ? 1 : 2;
         while (pl.tile_cols > 32 && copies * static_cast<size_t>(h->n) * pl.tile_cols * 4 > 76 * 1024) pl.tile_cols >>= 1;
       }
     } else {
@@ -286,7 +291,7 @@ int launch_regs(sgp_handle *h, const StepArgs &a, const Plan &pl, int64_t c0, in
   if (h->const_ok[static_cast<size_t>(slot)]) p.table_mode = 0;
   else p.table_mode = table_bytes <= 40 * 1024 ? 1 : 2;
   // large n: one exchange tile (two barriers per tile) so that the row segments can stay twice as long
-  p.single_buffer = h->n > 128 ? 1 : 0;
+  p.single_buffer = h->opt_single_buffer == 1 ? 1 : (h->opt_single_buffer == 2 ? 0 : (auto_single_buffer(h->n) ? 1 : 0));
   size_t smem = 0;
   for (;;) {
     smem = (p.single_buffer ? 1 : 2) * static_cast<size_t>(h->n) * tv * vec * 4 + 3 * static_cast<size_t>(h->n) * 4 +
@@ -755,6 +760,9 @@ int sgp_set_option(sgp_handle *h, const char *key, int64_t value) {
   } else if (std::strcmp(key, "stages") == 0) {
     if (value > 8) return SGP_ERR_ARG;
     h->opt_stages = value;
+  } else if (std::strcmp(key, "single_buffer") == 0) {
+    if (value > 2) return SGP_ERR_ARG;
+    h->opt_single_buffer = value;
   } else if (std::strcmp(key, "l2_hint") == 0) {
     if (value > 4) return SGP_ERR_ARG;
     h->opt_l2_hint = value;
@@ -771,6 +779,7 @@ int sgp_get_option(const sgp_handle *h, const char *key, int64_t *value) {
   else if (std::strcmp(key, "ctas_per_sm") == 0) *value = h->opt_ctas_per_sm;
   else if (std::strcmp(key, "stages") == 0) *value = h->opt_stages;
   else if (std::strcmp(key, "l2_hint") == 0) *value = h->opt_l2_hint;
+  else if (std::strcmp(key, "single_buffer") == 0) *value = h->opt_single_buffer;
   else if (std::strcmp(key, "last_variant") == 0) *value = h->last_variant;
   else if (std::strcmp(key, "last_grid") == 0) *value = h->last_grid;
   else if (std::strcmp(key, "last_smem") == 0) *value = h->last_smem;

@@ -417,3 +417,20 @@ def test_steps_can_be_captured_in_a_cuda_graph(binding, inputs, variant):
         assert h.device_status() == 0
     for a, b in ((X, X2), (W, W2), (M, M2), (Z, Z2)):
         assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("tau", [0, 1])
+@pytest.mark.parametrize("variant", [1, 3])
+def test_custom_weighted_schedule_on_gpu(binding, inputs, tau, variant):
+    """Per-edge, non-uniform mixing weights on an irregular time-varying digraph (three steps)."""
+    from test_schedule_compiler import _random_custom_schedule
+    from oracle import schedule as osched
+    n, steps = 12, 3
+    step, send, recv, wt = _random_custom_schedule(n, steps, seed=5)
+    g = binding.GraphDesc.custom(steps, step, send, recv, wt)
+    mats = [osched.custom_mixing_matrix(n, send[step == k], recv[step == k], wt[step == k].astype(np.float32))
+            for k in range(steps)]
+    w = inputs.Workload("custom", n=n, d=3000, K=11, graph="custom", lr=0.05, momentum=0.9, tau=tau)
+    out = _run_gpu(binding, inputs, w, graph=g, options={"variant": variant})
+    _compare(w, out, P_of_k=lambda k: mats[k % steps])
+    assert np.ptp(out["W"]) > 1e-2

@@ -162,3 +162,33 @@ def test_handle_calls_reject_null_without_a_gpu(binding):
     assert lib.sgp_create(C.byref(out), 4, 10, 8, C.byref(g.c), 0, 0) == binding.SGP_ERR_ARG      # ld < d
     assert lib.sgp_create(C.byref(out), 4, 10, 10, C.byref(g.c), -1, 0) == binding.SGP_ERR_ARG    # tau < 0
     assert out.value is None
+
+
+def _random_custom_schedule(n, steps, seed):
+    """Random column-stochastic schedule with NON-uniform fp32 weights (every column sums to 1 in fp32 exactly
+    enough for the compiler's check): per sender a random out-set incl. self and Dirichlet-like weights."""
+    rng = np.random.default_rng(seed)
+    step, send, recv, wt = [], [], [], []
+    for k in range(steps):
+        for j in range(n):
+            deg = int(rng.integers(0, min(5, n)))
+            targets = [j] + [int(t) for t in rng.choice([t for t in range(n) if t != j], size=deg, replace=False)]
+            raw = rng.random(len(targets)) + 0.1
+            w = (raw / raw.sum()).astype(np.float32)
+            w[0] = np.float32(1.0 - float(w[1:].astype(np.float64).sum()))        # make the fp32 column sum ~1
+            for t, p in zip(targets, w):
+                step.append(k); send.append(j); recv.append(t); wt.append(float(p))
+    perm = rng.permutation(len(step))                                             # any edge order is accepted
+    return [np.asarray(a)[perm] for a in (step, send, recv, wt)]
+
+
+@pytest.mark.parametrize("n,steps,seed", [(2, 1, 0), (7, 3, 1), (33, 4, 2), (256, 2, 3)])
+def test_custom_random_weighted_schedules_bit_exact(binding, n, steps, seed):
+    step, send, recv, wt = _random_custom_schedule(n, steps, seed)
+    sched = binding.Schedule(n, binding.GraphDesc.custom(steps, step, send, recv, wt))
+    assert sched.period == steps
+    for k in range(steps):
+        sel = step == k
+        P = S.custom_mixing_matrix(n, send[sel], recv[sel], wt[sel].astype(np.float32))
+        assert np.allclose(P.sum(axis=0), 1.0, atol=1e-6)
+        _assert_slot_equal(sched, k, P)
