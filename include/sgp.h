@@ -31,7 +31,8 @@ extern "C" {
 #define SGP_ERR_GRAPH    -2   /* schedule is not a valid column-stochastic digraph with self-loops    */
 #define SGP_ERR_CUDA     -3   /* a CUDA runtime call failed; see sgp_last_cuda_error                  */
 #define SGP_ERR_ALLOC    -4   /* host or device allocation failed                                     */
-#define SGP_ERR_STATE    -5   /* call not valid for this handle (e.g. ring export with tau = 0)       */
+#define SGP_ERR_STATE    -5   /* call not valid for this handle (ring export with tau = 0; the current
+                                 CUDA device is not the one the handle was created on)               */
 #define SGP_ERR_DEVICE   -6   /* a kernel reported a bounded wait that ran out (status word non-zero) */
 
 #define SGP_MAX_NODES 256     /* n <= 256: one CTA keeps all n rows of a column tile on chip          */
@@ -107,7 +108,15 @@ int sgp_create(sgp_handle **out, int n, int64_t d, int64_t ld, const sgp_graph_d
                unsigned flags);
 /* Frees everything the handle owns.  Synchronises the device.  NULL is accepted. */
 int sgp_destroy(sgp_handle *h);
-/* The handle's compiled schedule (owned by the handle; valid until sgp_destroy). */
+/*
+ * sgp_set_graph: replaces the handle's graph schedule (same n) from now on -- the hybrid schemes of
+ * Sec. 6.1 / Table 3 (AllReduce-like complete graph or two-peer graph for the first epochs, one-peer
+ * graph afterwards).  State, momentum and the delay ring are untouched: messages already in transit
+ * are still delivered.  Step k of later calls uses slot k mod (new period).  Synchronises the device.
+ * On error the handle keeps its current schedule.
+ */
+int sgp_set_graph(sgp_handle *h, const sgp_graph_desc *g);
+/* The handle's compiled schedule (owned by the handle; valid until sgp_destroy or sgp_set_graph). */
 int sgp_get_schedule(const sgp_handle *h, const sgp_schedule **s);
 
 /*

@@ -25,7 +25,7 @@ EXPORTS = [
     "sgp_create", "sgp_destroy", "sgp_get_schedule", "sgp_step", "sgp_debias", "sgp_step_host", "sgp_reset",
     "sgp_ring_export", "sgp_ring_import", "sgp_check", "sgp_set_option", "sgp_get_option", "sgp_device_status",
     "sgp_last_cuda_error", "sgp_strerror", "sgp_version", "sgp_step_static",
-    "sgp_step_adam", "sgp_param_deviation",
+    "sgp_step_adam", "sgp_param_deviation", "sgp_set_graph",
 ]
 
 
@@ -61,6 +61,7 @@ def _load() -> C.CDLL:
         "sgp_create": [C.POINTER(vp), i32, i64, i64, C.POINTER(sgp_graph_desc), i32, C.c_uint],
         "sgp_destroy": [vp],
         "sgp_get_schedule": [vp, C.POINTER(vp)],
+        "sgp_set_graph": [vp, C.POINTER(sgp_graph_desc)],
         "sgp_step": [vp, vp, vp, vp, vp, vp, i64, f32, f32, f32, i32, vp],
         "sgp_debias": [vp, vp, vp, vp, vp],
         "sgp_step_adam": [vp, vp, vp, vp, vp, vp, vp, i64, i64, f32, f32, f32, f32, f32, vp],
@@ -216,6 +217,10 @@ class Sgp:
 
     def __exit__(self, *exc):
         self.close()
+
+    def set_graph(self, graph: GraphDesc) -> None:
+        """Switches the mixing schedule (hybrid schemes: dense mixing early, sparse later)."""
+        _check(_lib.sgp_set_graph(self._h, C.byref(graph.c)), "sgp_set_graph")
 
     @property
     def schedule(self) -> _ScheduleView:

@@ -8,6 +8,7 @@
 #include <map>
 #include <mutex>
 #include <new>
+#include <utility>
 #include <vector>
 
 #include "aux_kernels.cuh"
@@ -102,18 +103,19 @@ struct KernelInfo {
   size_t enabled_smem = 48 * 1024;
 };
 std::mutex g_kernel_info_mutex;
-std::map<const void *, KernelInfo> g_kernel_info;
+std::map<std::pair<int, const void *>, KernelInfo> g_kernel_info;   // function attributes are per device
 
 int kernel_info(sgp_handle *h, const void *kern, size_t smem, KernelInfo *out) {
   std::lock_guard<std::mutex> lock(g_kernel_info_mutex);
-  auto it = g_kernel_info.find(kern);
+  const std::pair<int, const void *> key(h->device, kern);
+  auto it = g_kernel_info.find(key);
   if (it == g_kernel_info.end()) {
     cudaFuncAttributes fa;
     SGP_CUDA_TRY(h, cudaFuncGetAttributes(&fa, kern));
     KernelInfo ki;
     ki.num_regs = fa.numRegs;
     ki.static_smem = fa.sharedSizeBytes;
-    it = g_kernel_info.emplace(kern, ki).first;
+    it = g_kernel_info.emplace(key, ki).first;
   }
   if (smem > it->second.enabled_smem) {
     SGP_CUDA_TRY(h, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
@@ -454,10 +456,80 @@ int launch_step_range(sgp_handle *h, const StepArgs &a, int64_t c0, int64_t c1, 
   return SGP_OK;
 }
 
+// The handle's tables and ring live on the device that was current at sgp_create.
+int check_device(const sgp_handle *h) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return SGP_ERR_CUDA;
+  }
+  return dev == h->device ? SGP_OK : SGP_ERR_STATE;
+}
+
 int validate_step(const sgp_handle *h, const float *X, const float *W, const float *M, const float *G, int64_t k,
                   float momentum) {
   if (h == nullptr || X == nullptr || W == nullptr || G == nullptr || k < 0) return SGP_ERR_ARG;
   if (momentum != 0.0f && M == nullptr) return SGP_ERR_ARG;
+  return check_device(h);
+}
+
+// Builds the device tables of a compiled schedule and installs them (and the schedule) in the handle,
+// releasing whatever the handle held before.  The caller guarantees that no kernel still reads the old tables.
+int upload_schedule(sgp_handle *h, sgp_schedule *sched) {
+  std::vector<int32_t> rowptr, col;
+  std::vector<float> val;
+  std::vector<int64_t> off_rowptr, off_nnz;
+  std::vector<ConstTable> const_tables;
+  std::vector<char> const_ok;
+  for (int64_t s = 0; s < sched->period(); ++s) {
+    const SgpStepCsr &c = sched->steps[static_cast<size_t>(s)];
+    off_rowptr.push_back(static_cast<int64_t>(rowptr.size()));
+    off_nnz.push_back(static_cast<int64_t>(col.size()));
+    rowptr.insert(rowptr.end(), c.rowptr.begin(), c.rowptr.end());
+    col.insert(col.end(), c.col.begin(), c.col.end());
+    val.insert(val.end(), c.val.begin(), c.val.end());
+    ConstTable ct{};
+    const bool fits = h->n <= sgp::kConstRows && static_cast<int>(c.col.size()) <= sgp::kConstNnz;
+    if (fits) {
+      std::copy(c.rowptr.begin(), c.rowptr.end(), ct.rowptr);
+      std::copy(c.col.begin(), c.col.end(), ct.col);
+      std::copy(c.val.begin(), c.val.end(), ct.val);
+    }
+    const_tables.push_back(ct);
+    const_ok.push_back(fits ? 1 : 0);
+  }
+  int32_t *d_rowptr = nullptr, *d_col = nullptr;
+  float *d_val = nullptr;
+  auto release = [&]() {
+    cudaFree(d_rowptr);
+    cudaFree(d_col);
+    cudaFree(d_val);
+    (void)cudaGetLastError();
+  };
+  if (cudaMalloc(&d_rowptr, rowptr.size() * sizeof(int32_t)) != cudaSuccess ||
+      cudaMalloc(&d_col, col.size() * sizeof(int32_t)) != cudaSuccess ||
+      cudaMalloc(&d_val, val.size() * sizeof(float)) != cudaSuccess) {
+    release();
+    return SGP_ERR_ALLOC;
+  }
+  if (cudaMemcpy(d_rowptr, rowptr.data(), rowptr.size() * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(d_col, col.data(), col.size() * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(d_val, val.data(), val.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess) {
+    release();
+    return SGP_ERR_CUDA;
+  }
+  cudaFree(h->d_rowptr);
+  cudaFree(h->d_col);
+  cudaFree(h->d_val);
+  h->d_rowptr = d_rowptr;
+  h->d_col = d_col;
+  h->d_val = d_val;
+  h->off_rowptr.swap(off_rowptr);
+  h->off_nnz.swap(off_nnz);
+  h->const_tables.swap(const_tables);
+  h->const_ok.swap(const_ok);
+  if (h->sched != sched) delete h->sched;
+  h->sched = sched;
   return SGP_OK;
 }
 
@@ -514,33 +586,10 @@ int sgp_create(sgp_handle **out, int n, int64_t d, int64_t ld, const sgp_graph_d
   e = cudaDeviceGetAttribute(&h->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, h->device);
   if (e != cudaSuccess) return fail(SGP_ERR_CUDA, e);
 
-  // concatenate the slots and upload
-  std::vector<int32_t> rowptr, col;
-  std::vector<float> val;
-  const int64_t period = sched->period();
-  for (int64_t s = 0; s < period; ++s) {
-    const SgpStepCsr &c = sched->steps[static_cast<size_t>(s)];
-    h->off_rowptr.push_back(static_cast<int64_t>(rowptr.size()));
-    h->off_nnz.push_back(static_cast<int64_t>(col.size()));
-    rowptr.insert(rowptr.end(), c.rowptr.begin(), c.rowptr.end());
-    col.insert(col.end(), c.col.begin(), c.col.end());
-    val.insert(val.end(), c.val.begin(), c.val.end());
-    ConstTable ct{};
-    const bool fits = n <= sgp::kConstRows && static_cast<int>(c.col.size()) <= sgp::kConstNnz;
-    if (fits) {
-      std::copy(c.rowptr.begin(), c.rowptr.end(), ct.rowptr);
-      std::copy(c.col.begin(), c.col.end(), ct.col);
-      std::copy(c.val.begin(), c.val.end(), ct.val);
-    }
-    h->const_tables.push_back(ct);
-    h->const_ok.push_back(fits ? 1 : 0);
+  {
+    const int rc_up = upload_schedule(h, sched);
+    if (rc_up != SGP_OK) return fail(rc_up, cudaSuccess);
   }
-  e = cudaMalloc(&h->d_rowptr, rowptr.size() * sizeof(int32_t));
-  if (e != cudaSuccess) return fail(SGP_ERR_ALLOC, e);
-  e = cudaMalloc(&h->d_col, col.size() * sizeof(int32_t));
-  if (e != cudaSuccess) return fail(SGP_ERR_ALLOC, e);
-  e = cudaMalloc(&h->d_val, val.size() * sizeof(float));
-  if (e != cudaSuccess) return fail(SGP_ERR_ALLOC, e);
   e = cudaMalloc(&h->d_words, 2 * sizeof(unsigned));
   if (e != cudaSuccess) return fail(SGP_ERR_ALLOC, e);
   e = cudaMalloc(&h->d_stats, (4 + SGP_MAX_NODES) * sizeof(double));
@@ -555,12 +604,6 @@ int sgp_create(sgp_handle **out, int n, int64_t d, int64_t ld, const sgp_graph_d
     e = cudaMemset(h->ring_w, 0, static_cast<size_t>(tau) * n * sizeof(float));
     if (e != cudaSuccess) return fail(SGP_ERR_CUDA, e);
   }
-  e = cudaMemcpy(h->d_rowptr, rowptr.data(), rowptr.size() * sizeof(int32_t), cudaMemcpyHostToDevice);
-  if (e != cudaSuccess) return fail(SGP_ERR_CUDA, e);
-  e = cudaMemcpy(h->d_col, col.data(), col.size() * sizeof(int32_t), cudaMemcpyHostToDevice);
-  if (e != cudaSuccess) return fail(SGP_ERR_CUDA, e);
-  e = cudaMemcpy(h->d_val, val.data(), val.size() * sizeof(float), cudaMemcpyHostToDevice);
-  if (e != cudaSuccess) return fail(SGP_ERR_CUDA, e);
   e = cudaMemset(h->d_words, 0, 2 * sizeof(unsigned));
   if (e != cudaSuccess) return fail(SGP_ERR_CUDA, e);
   e = cudaDeviceSynchronize();
@@ -574,6 +617,19 @@ int sgp_destroy(sgp_handle *h) {
   (void)cudaDeviceSynchronize();
   free_handle(h);
   return SGP_OK;
+}
+
+int sgp_set_graph(sgp_handle *h, const sgp_graph_desc *g) {
+  if (h == nullptr || g == nullptr) return SGP_ERR_ARG;
+  int rc = check_device(h);
+  if (rc != SGP_OK) return rc;
+  sgp_schedule *sched = nullptr;
+  rc = sgp_schedule_build(&sched, h->n, g);
+  if (rc != SGP_OK) return rc;                       // the handle keeps its current schedule
+  SGP_CUDA_TRY(h, cudaDeviceSynchronize());          // no kernel may still read the old tables
+  rc = upload_schedule(h, sched);
+  if (rc != SGP_OK) delete sched;
+  return rc;
 }
 
 int sgp_get_schedule(const sgp_handle *h, const sgp_schedule **s) {
@@ -596,6 +652,7 @@ int sgp_step_adam(sgp_handle *h, float *d_X, float *d_W, float *d_M1, float *d_M
   if (h == nullptr || d_X == nullptr || d_W == nullptr || d_M1 == nullptr || d_M2 == nullptr || d_G == nullptr ||
       k < 0 || t < 1 || !(beta1 >= 0.0f && beta1 < 1.0f) || !(beta2 >= 0.0f && beta2 < 1.0f) || !(eps >= 0.0f))
     return SGP_ERR_ARG;
+  if (check_device(h) != SGP_OK) return check_device(h);
   StepArgs a{d_X, d_W, d_M1, d_G, d_Z, k, lr, 0.0f, weight_decay, sgp::kUpdAdam};
   a.V = d_M2;
   a.beta1 = beta1;

@@ -119,8 +119,8 @@ __device__ __forceinline__ V local_update(V x, V g, V &u, V &v, const StepParams
   return vfma(-p.lr, s, x);
 }
 
-// Shared-memory carve-up (dynamic): [H tile: tile_items vectors][w_old n][rw_in n][inv_w n][p_self n]
-// then the CSR copy when table_mode < 2.
+// Per-CTA scratch after the tiles/stages in dynamic shared memory: [w_old n][rw_in n][inv_w n], then the
+// CSR copy [rowptr n+1][col nnz][val nnz] when table_mode < 2.
 struct CtaTables {
   const int32_t *rowptr;
   const int32_t *col;

@@ -434,3 +434,37 @@ def test_custom_weighted_schedule_on_gpu(binding, inputs, tau, variant):
     out = _run_gpu(binding, inputs, w, graph=g, options={"variant": variant})
     _compare(w, out, P_of_k=lambda k: mats[k % steps])
     assert np.ptp(out["W"]) > 1e-2
+
+
+@pytest.mark.parametrize("first,tau", [("complete", 0), ("two_peer", 0), ("two_peer", 2)])
+def test_hybrid_schedules_switch_graph_mid_run(binding, inputs, first, tau):
+    """AR/1P-SGP and 2P/1P-SGP (Table 3): dense mixing for the first steps, one-peer graph afterwards."""
+    from oracle import schedule as osched
+    n, d, K, K1 = 16, 3000, 14, 5
+    w = inputs.Workload("hybrid", n=n, d=d, K=K, graph="exp", peers=1, lr=0.1, momentum=0.9, weight_decay=1e-4, tau=tau)
+    g_first = binding.GraphDesc.complete() if first == "complete" else binding.GraphDesc.exp_peers(2)
+    def P_of_k(k):
+        if k < K1:
+            return osched.mixing_matrix("complete", n, k) if first == "complete" else osched.mixing_matrix("exp", n, k, peers=2)
+        return osched.mixing_matrix("exp", n, k, peers=1)
+    X = inputs.initial_x(w, device=DEV).contiguous(); W = torch.ones(n, device=DEV)
+    M = torch.zeros((n, d), device=DEV); Z = torch.empty((n, d), device=DEV); G = torch.empty((n, d), device=DEV)
+    x0 = X.cpu().numpy().copy(); grads = []
+    with binding.Sgp(n, d, g_first, tau=tau) as h:
+        for k in range(K):
+            if k == K1:
+                h.set_graph(binding.GraphDesc.exp_peers(1))
+                assert h.schedule.period == 4
+            grads.append(inputs.gradient(w, k, G).cpu().numpy().copy())
+            h.step(X, W, M, G, Z, k, w.lr, w.momentum, w.weight_decay, True)
+        torch.cuda.synchronize()
+        with pytest.raises(binding.SgpError):
+            h.set_graph(binding.GraphDesc.exp_peers(0))             # rejected: the old schedule stays
+        assert h.schedule.period == 4
+        out = dict(x0=x0, grads=grads, X=X.cpu().numpy(), W=W.cpu().numpy(), M=M.cpu().numpy(), Z=Z.cpu().numpy(),
+                   stats=h.check(X, W), ring=None)
+        if tau:
+            rx = torch.empty((tau, n, d), device=DEV); rw = torch.empty((tau, n), device=DEV)
+            h.ring_export(rx, rw); torch.cuda.synchronize()
+            out["ring"] = (rx.cpu().numpy(), rw.cpu().numpy())
+    _compare(w, out, P_of_k=P_of_k)
