@@ -205,6 +205,10 @@ int sgp_param_deviation(sgp_handle *h, const float *d_A, double *h_dev, void *st
  *   "stages"       shared-memory stages of the bulk-copy pipeline (0 = automatic, at most 8)
  *   "single_buffer" register-staged kernel: 0 = automatic (n > 128), 1 = one exchange tile and two barriers
  *                  per tile, 2 = two exchange tiles and one barrier
+ *   "wait_limit_ms" bound of every in-kernel wait of the pipelined kernel (0 = 2000 ms); a wait that runs out
+ *                  sets the device status word (sgp_device_status) and the CTA leaves: nothing hangs
+ *   "inject_stall" test hook, 0/1: one CTA of the pipelined kernel never requests its first tile, so that
+ *                  the bounded wait and the status word can be exercised (that step's results are invalid)
  *   "l2_hint"      L2 evict-first policy on the pipeline's bulk copies: 0 = automatic (gradients only),
  *                  1 = every array, 2 = none, 3 = gradients only, 4 = every array but the gradients
  * Read-only through sgp_get_option: "last_variant", "last_grid", "last_smem", "last_tile_cols" describe
@@ -244,7 +248,9 @@ int sgp_step_static(int n, int64_t d, int64_t ld, const int32_t *h_rowptr, const
                     const float *h_val, int64_t nnz, float *d_X, float *d_W, float *d_M, const float *d_G,
                     float *d_Z, float lr, float momentum, float weight_decay, int nesterov, void *stream);
 
-/* Reads the handle's device status word (0 = no kernel ever gave up a bounded wait).  Synchronises. */
+/* Reads the handle's device status word (0 = no kernel ever gave up a bounded wait; bit 0: consumers gave up
+ * waiting for a tile, bit 1: the producer gave up waiting for a free stage, bit 2: copies were still
+ * pending at exit).  sgp_reset clears it.  Synchronises. */
 int sgp_device_status(sgp_handle *h, unsigned *status);
 /* cudaError_t value latched by the last call that returned SGP_ERR_CUDA on this handle (0 if none). */
 int sgp_last_cuda_error(const sgp_handle *h);

@@ -39,7 +39,8 @@ struct sgp_handle {
   float *ring_w = nullptr;   // tau * n
   unsigned *d_words = nullptr;  // [0] ticket, [1] status
   double *d_stats = nullptr;    // 4 doubles for sgp_check, then SGP_MAX_NODES doubles for sgp_param_deviation
-  int64_t opt_variant = 0, opt_tile_cols = 0, opt_ctas_per_sm = 0, opt_stages = 0, opt_l2_hint = 0, opt_single_buffer = 0;
+  int64_t opt_variant = 0, opt_tile_cols = 0, opt_ctas_per_sm = 0, opt_stages = 0, opt_l2_hint = 0, opt_single_buffer = 0, opt_wait_limit_ms = 0,
+          opt_inject_stall = 0;
   int64_t last_variant = 0, last_grid = 0, last_smem = 0, last_tile_cols = 0;   // of the most recent step launch
   cudaStream_t s_h2d = nullptr, s_compute = nullptr, s_d2h = nullptr;
   std::vector<cudaEvent_t> ev_in, ev_done;
@@ -404,6 +405,8 @@ int launch_tma(sgp_handle *h, const StepArgs &a, const Plan &pl, int64_t c0, int
   const int64_t tile_cols = tv * 4;
   const int64_t ntiles = (c1 - c0 + tile_cols - 1) / tile_cols;
   const int64_t grid = std::min<int64_t>(ntiles, static_cast<int64_t>(h->sm_count) * cps);
+  p.wait_limit_ms = h->opt_wait_limit_ms > 0 ? static_cast<int>(h->opt_wait_limit_ms) : 2000;
+  p.inject_stall = h->opt_inject_stall ? 1 : 0;
   p.l2_hint = h->opt_l2_hint == 2 ? 0 : (h->opt_l2_hint == 0 ? 3 : static_cast<int>(h->opt_l2_hint));
   TmaKernel kern = pick_tma(a.upd, a.Z != nullptr, has_ring);
   {
@@ -817,6 +820,12 @@ int sgp_set_option(sgp_handle *h, const char *key, int64_t value) {
   } else if (std::strcmp(key, "stages") == 0) {
     if (value > 8) return SGP_ERR_ARG;
     h->opt_stages = value;
+  } else if (std::strcmp(key, "wait_limit_ms") == 0) {
+    if (value > 10000) return SGP_ERR_ARG;
+    h->opt_wait_limit_ms = value;
+  } else if (std::strcmp(key, "inject_stall") == 0) {
+    if (value > 1) return SGP_ERR_ARG;
+    h->opt_inject_stall = value;
   } else if (std::strcmp(key, "single_buffer") == 0) {
     if (value > 2) return SGP_ERR_ARG;
     h->opt_single_buffer = value;
@@ -837,6 +846,8 @@ int sgp_get_option(const sgp_handle *h, const char *key, int64_t *value) {
   else if (std::strcmp(key, "stages") == 0) *value = h->opt_stages;
   else if (std::strcmp(key, "l2_hint") == 0) *value = h->opt_l2_hint;
   else if (std::strcmp(key, "single_buffer") == 0) *value = h->opt_single_buffer;
+  else if (std::strcmp(key, "wait_limit_ms") == 0) *value = h->opt_wait_limit_ms;
+  else if (std::strcmp(key, "inject_stall") == 0) *value = h->opt_inject_stall;
   else if (std::strcmp(key, "last_variant") == 0) *value = h->last_variant;
   else if (std::strcmp(key, "last_grid") == 0) *value = h->last_grid;
   else if (std::strcmp(key, "last_smem") == 0) *value = h->last_smem;

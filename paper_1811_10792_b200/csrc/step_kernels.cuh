@@ -44,6 +44,9 @@ struct StepParams {
   int l2_hint;         // TMA kernel, L2 evict-first policy on the bulk copies: 0 none, 1 every array, 3 only G
                        // (dead after its read; X, M, V, ring are rewritten in place and keep the normal
                        // policy: measured 0.985 of the copy bandwidth against 0.967 without), 4 all but G
+  int wait_limit_ms;   // TMA kernel: bound of every mbarrier wait in milliseconds
+  int inject_stall;    // TMA kernel, fault-injection for tests: CTA 0 never requests its first tile, so its
+                       // consumers' bounded wait runs out and the status word is set (nothing hangs)
   float lr, momentum, wd;
   // Adam only: decay rates, epsilon, lr / (1 - beta1^t) and 1 / sqrt(1 - beta2^t)
   float beta1, beta2, eps, adam_step, adam_rsqrt_bc2;
@@ -350,15 +353,15 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-// Waits for the phase with the given parity; gives up after about two seconds.
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity) {
+// Waits for the phase with the given parity; gives up after limit_ns (wall clock of the device).
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity, uint64_t limit_ns) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_timer_ns();
   for (;;) {
 #pragma unroll 1
     for (int i = 0; i < 256; ++i)
       if (mbar_try_wait(bar, parity)) return true;
-    if (global_timer_ns() - t0 > 2000000000ull) return false;
+    if (global_timer_ns() - t0 > limit_ns) return false;
   }
 }
 // One contiguous global -> shared copy of `bytes` (multiple of 16, both addresses 16-byte aligned).
@@ -447,6 +450,7 @@ sgp_step_tma_kernel(const __grid_constant__ StepParams p, const __grid_constant_
   const int64_t my_tiles = ntiles > blockIdx.x ? (ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int *abort_flag = &s_abort;
+  const uint64_t limit_ns = static_cast<uint64_t>(p.wait_limit_ms) * 1000000ull;
 
   if (warp == kTmaConsumers / 32) {
     // ---------------- producer warp
@@ -455,11 +459,12 @@ sgp_step_tma_kernel(const __grid_constant__ StepParams p, const __grid_constant_
     for (int64_t it = 0; it < my_tiles && !*abort_flag; ++it) {
       const int s = static_cast<int>(it % stages);
       const int64_t round = it / stages;
-      if (round > 0 && !mbar_wait_bounded(empty_bar + s, static_cast<uint32_t>((round - 1) & 1))) {
+      if (round > 0 && !mbar_wait_bounded(empty_bar + s, static_cast<uint32_t>((round - 1) & 1), limit_ns)) {
         if (lane == 0) atomicOr(p.status, kStatusEmptyTimeout);
         *abort_flag = 1;
         break;
       }
+      if (p.inject_stall && blockIdx.x == 0 && it == 0) continue;   // test hook: this tile is never requested
       const int64_t tile = blockIdx.x + it * gridDim.x;
       const int64_t col0 = p.col_begin + tile * tile_cols;
       const int64_t valid = min(tile_cols, p.col_end - col0);
@@ -499,8 +504,9 @@ sgp_step_tma_kernel(const __grid_constant__ StepParams p, const __grid_constant_
     // On an aborted run copies may still be in flight to this CTA's shared memory: wait for them (bounded).
     if (*abort_flag) {
       for (int64_t it = (issued > stages ? issued - stages : 0); it < issued; ++it) {
+        if (p.inject_stall && blockIdx.x == 0 && it == 0) continue;   // was never requested
         const int s = static_cast<int>(it % stages);
-        if (!mbar_wait_bounded(full_bar + s, static_cast<uint32_t>((it / stages) & 1)) && lane == 0)
+        if (!mbar_wait_bounded(full_bar + s, static_cast<uint32_t>((it / stages) & 1), limit_ns) && lane == 0)
           atomicOr(p.status, kStatusDrainTimeout);
       }
     }
@@ -511,7 +517,7 @@ sgp_step_tma_kernel(const __grid_constant__ StepParams p, const __grid_constant_
       const int s = static_cast<int>(it % stages);
       const int64_t round = it / stages;
       // bounded wait, then a vote: either every consumer goes on or every consumer leaves
-      const bool arrived = !*abort_flag && mbar_wait_bounded(full_bar + s, static_cast<uint32_t>(round & 1));
+      const bool arrived = !*abort_flag && mbar_wait_bounded(full_bar + s, static_cast<uint32_t>(round & 1), limit_ns);
       if (!consumer_all(arrived)) {
         if (ctid == 0) atomicOr(p.status, kStatusFullTimeout);
         *abort_flag = 1;

@@ -468,3 +468,39 @@ def test_hybrid_schedules_switch_graph_mid_run(binding, inputs, first, tau):
             h.ring_export(rx, rw); torch.cuda.synchronize()
             out["ring"] = (rx.cpu().numpy(), rw.cpu().numpy())
     _compare(w, out, P_of_k=P_of_k)
+
+
+def test_bounded_wait_reports_status_instead_of_hanging(binding, inputs):
+    """Failure detection without a fault: one CTA's tile is never requested, its consumers' wait runs out after
+    the configured bound, the kernel returns, the status word says so, and the handle keeps working."""
+    import time
+    w = inputs.WORKLOADS["resnet50"].scaled(256 * 600, K=1)
+    n, d = w.n, w.d
+    def state():
+        X = inputs.initial_x(w, device=DEV).contiguous()
+        return X, torch.ones(n, device=DEV), torch.zeros((n, d), device=DEV), torch.empty((n, d), device=DEV)
+    G = inputs.gradient(w, 0, torch.empty((n, d), device=DEV))
+    with binding.Sgp(n, d, graph_desc(w, binding)) as h:
+        h.set_option("variant", 3)
+        h.set_option("wait_limit_ms", 200)
+        h.set_option("inject_stall", 1)
+        X, W, M, Z = state()
+        t0 = time.perf_counter()
+        h.step(X, W, M, G, Z, 0, w.lr, w.momentum, 0.0, True)
+        torch.cuda.synchronize()                                   # returns: no hang, no CUDA error
+        assert time.perf_counter() - t0 < 5.0
+        assert h.get_option("last_variant") == 3
+        status = h.device_status()
+        assert status & 1                                          # consumers gave up on the missing tile
+        h.reset()
+        h.set_option("inject_stall", 0)
+        assert h.device_status() == 0
+        X, W, M, Z = state()
+        h.step(X, W, M, G, Z, 0, w.lr, w.momentum, 0.0, True)     # the context and the handle are still usable
+        torch.cuda.synchronize()
+        assert h.device_status() == 0
+        ref = state()
+        h.set_option("variant", 1)
+        h.step(ref[0], ref[1], ref[2], G, ref[3], 0, w.lr, w.momentum, 0.0, True)
+        torch.cuda.synchronize()
+        assert torch.equal(X, ref[0]) and torch.equal(Z, ref[3]) and torch.equal(M, ref[2])
