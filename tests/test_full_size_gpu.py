@@ -80,21 +80,56 @@ def _run_full(binding, inputs, w, K, ld_align=256):
 
 @pytest.mark.parametrize("ld_align", [256, 1])
 def test_resnet50_full_size(binding, inputs, ld_align):
-    _run_full(binding, inputs, inputs.WORKLOADS["resnet50"], K=3, ld_align=ld_align)
+    _run_full(binding, inputs, inputs.WORKLOADS["resnet50"], K=20 if ld_align == 256 else 3, ld_align=ld_align)
 
 
 def test_transformer_full_size(binding, inputs):
-    _run_full(binding, inputs, inputs.WORKLOADS["transformer"], K=3)
+    _run_full(binding, inputs, inputs.WORKLOADS["transformer"], K=20)
 
 
 def test_resnet50_overlap_full_size(binding, inputs):
-    _run_full(binding, inputs, inputs.WORKLOADS["resnet50_osgp1"], K=3)
+    _run_full(binding, inputs, inputs.WORKLOADS["resnet50_osgp1"], K=20)
 
 
 @pytest.mark.parametrize("n,d", [(256, 10_000_000), (64, 100_000_000)])
 def test_sweep_largest_points(binding, inputs, n, d):
     """More than 2^31 elements per array: 64-bit offsets everywhere."""
     _run_full(binding, inputs, inputs.sweep_workload(n, d), K=2)
+
+
+def test_transformer_adam_full_size(binding, inputs):
+    """Adam-SGP at the Transformer size, K = 5 steps, sampled windows."""
+    from oracle import sgp as osgp
+    from parity_util import oracle_P_of_k
+    w = inputs.WORKLOADS["transformer_adam"]
+    n, d, K = w.n, w.d, 5
+    X, ld = binding.empty_matrix(n, d, device=DEV)
+    X.copy_(inputs.initial_x(w, device=DEV))
+    M1, _ = binding.empty_matrix(n, d, device=DEV, fill=0.0)
+    M2, _ = binding.empty_matrix(n, d, device=DEV, fill=0.0)
+    Z, _ = binding.empty_matrix(n, d, device=DEV, fill=float("nan"))
+    G, _ = binding.empty_matrix(n, d, device=DEV)
+    W = torch.ones(n, device=DEV)
+    wins = _windows(d)
+    x0 = [X[:, a:b].cpu().numpy().copy() for a, b in wins]
+    grads = [[] for _ in wins]
+    with binding.Sgp(n, d, graph_desc(w, binding), ld=ld) as h:
+        for k in range(K):
+            inputs.gradient(w, k, G)
+            for i, (a, b) in enumerate(wins):
+                grads[i].append(G[:, a:b].cpu().numpy().copy())
+            h.step_adam(X, W, M1, M2, G, Z, k, k + 1, w.lr, w.beta1, w.beta2, w.adam_eps, 0.0)
+        torch.cuda.synchronize()
+        assert h.device_status() == 0
+    for i, (a, b) in enumerate(wins):
+        st = osgp.sgp_run(x0[i].astype(np.float64), K, oracle_P_of_k(w), lambda k, z: grads[i][k].astype(np.float64),
+                          w.lr, adam=(w.beta1, w.beta2, w.adam_eps))
+        assert_close(f"X[{a}:{b}]", X[:, a:b].cpu().numpy(), st.x)
+        assert_close(f"Z[{a}:{b}]", Z[:, a:b].cpu().numpy(), st.z)
+        assert_close(f"M1[{a}:{b}]", M1[:, a:b].cpu().numpy(), st.u)
+        assert_close(f"M2[{a}:{b}]", M2[:, a:b].cpu().numpy(), st.v)
+    del X, M1, M2, Z, G
+    torch.cuda.empty_cache()
 
 
 def test_tau_full_size_mass_conservation(binding, inputs):
