@@ -356,6 +356,7 @@ def main():
         dist.barrier()
     torch.cuda.synchronize()
     evs = [torch.cuda.Event(enable_timing=True) for _ in range(K + 1)]
+    launches_before = h.get_option("launches")
     sampler.arm(True)
     for i in range(K):
         evs[i].record()
@@ -365,6 +366,7 @@ def main():
     sampler.arm(False)
     if world > 1:
         dist.barrier()
+    gpu_launches = h.get_option("launches") - launches_before      # step kernels launched inside the timed region
     total_ms = evs[0].elapsed_time(evs[K])
     per_step_ms = [evs[i].elapsed_time(evs[i + 1]) for i in range(K)]
     assert h.device_status() == 0
@@ -418,7 +420,8 @@ def main():
             "dtype": "f32", "data": "synthetic",
             "config": workload_config(w, extra={"gradient_pool": pool, "parallelism": f"replicas x{world}",
                                                 "row_pitch_floats": ld}),
-            "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": K, "clocks": sampler.summary(),
+            "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": gpu_launches,
+            "clocks": sampler.summary(),
         }
         print(json.dumps(line), flush=True)
     h.close()

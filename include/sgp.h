@@ -212,7 +212,8 @@ int sgp_param_deviation(sgp_handle *h, const float *d_A, double *h_dev, void *st
  *   "l2_hint"      L2 evict-first policy on the pipeline's bulk copies: 0 = automatic (gradients only),
  *                  1 = every array, 2 = none, 3 = gradients only, 4 = every array but the gradients
  * Read-only through sgp_get_option: "last_variant", "last_grid", "last_smem", "last_tile_cols" describe
- * the most recent step launch of the handle (which kernel ran, CTAs, dynamic shared memory, tile width).
+ * the most recent step launch of the handle (which kernel ran, CTAs, dynamic shared memory, tile width);
+ * "launches" counts the step kernels the handle has launched so far.
  * Unknown keys or unsupported values return SGP_ERR_ARG and change nothing.
  */
 int sgp_set_option(sgp_handle *h, const char *key, int64_t value);

@@ -42,6 +42,7 @@ struct sgp_handle {
   int64_t opt_variant = 0, opt_tile_cols = 0, opt_ctas_per_sm = 0, opt_stages = 0, opt_l2_hint = 0, opt_single_buffer = 0, opt_wait_limit_ms = 0,
           opt_inject_stall = 0;
   int64_t last_variant = 0, last_grid = 0, last_smem = 0, last_tile_cols = 0;   // of the most recent step launch
+  int64_t launches = 0;                                                          // step kernels launched so far
   cudaStream_t s_h2d = nullptr, s_compute = nullptr, s_d2h = nullptr;
   std::vector<cudaEvent_t> ev_in, ev_done;
   int last_cuda_error = 0;
@@ -329,6 +330,7 @@ int launch_regs(sgp_handle *h, const StepArgs &a, const Plan &pl, int64_t c0, in
   kern<<<static_cast<unsigned>(grid), sgp::kThreads, smem, stream>>>(p, ct);
   SGP_CUDA_TRY(h, cudaGetLastError());
   h->last_variant = 1;
+  ++h->launches;
   h->last_grid = grid;
   h->last_smem = static_cast<int64_t>(smem);
   h->last_tile_cols = tile_cols;
@@ -428,6 +430,7 @@ int launch_tma(sgp_handle *h, const StepArgs &a, const Plan &pl, int64_t c0, int
   kern<<<static_cast<unsigned>(grid), sgp::kTmaThreads, smem, stream>>>(p, ct, maps, stages, use_maps ? 1 : 0);
   SGP_CUDA_TRY(h, cudaGetLastError());
   h->last_variant = use_maps ? 2 : 3;
+  ++h->launches;
   h->last_grid = grid;
   h->last_smem = static_cast<int64_t>(smem);
   h->last_tile_cols = tile_cols;
@@ -850,6 +853,7 @@ int sgp_get_option(const sgp_handle *h, const char *key, int64_t *value) {
   else if (std::strcmp(key, "inject_stall") == 0) *value = h->opt_inject_stall;
   else if (std::strcmp(key, "last_variant") == 0) *value = h->last_variant;
   else if (std::strcmp(key, "last_grid") == 0) *value = h->last_grid;
+  else if (std::strcmp(key, "launches") == 0) *value = h->launches;
   else if (std::strcmp(key, "last_smem") == 0) *value = h->last_smem;
   else if (std::strcmp(key, "last_tile_cols") == 0) *value = h->last_tile_cols;
   else return SGP_ERR_ARG;
