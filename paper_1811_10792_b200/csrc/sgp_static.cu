@@ -105,12 +105,16 @@ int launch(const DeviceSetup &s, sgp::StepParams p, int vec, int64_t c0, int64_t
     (void)cudaGetLastError();
     return SGP_ERR_CUDA;
   }
-  int resident = 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, reinterpret_cast<const void *>(kern), sgp::kThreads,
-                                                    smem) != cudaSuccess) {
+  // CTAs resident per SM by registers, shared memory and threads: the grid is exactly one wave
+  cudaFuncAttributes fa;
+  if (cudaFuncGetAttributes(&fa, reinterpret_cast<const void *>(kern)) != cudaSuccess) {
     (void)cudaGetLastError();
     return SGP_ERR_CUDA;
   }
+  const int regs_per_cta = ((fa.numRegs + 7) / 8 * 8) * sgp::kThreads;
+  const int resident = std::min({regs_per_cta > 0 ? 65536 / regs_per_cta : 8,
+                                 static_cast<int>((227 * 1024) / (smem + fa.sharedSizeBytes + 1024)),
+                                 2048 / sgp::kThreads});
   const int64_t tile_cols = (int64_t{1} << log2_tv) * vec;
   const int64_t ntiles = (c1 - c0 + tile_cols - 1) / tile_cols;
   const int64_t grid = std::min<int64_t>(ntiles, static_cast<int64_t>(s.sm_count) * std::max(1, resident));
