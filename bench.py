@@ -30,12 +30,12 @@ UNIT = "updates/s"
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused step kernel, from the ncu capture
-# summarised under profiles/ (captured on a column-scaled case and scaled by the units processed).
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused step kernel, from one ncu capture of the
+# same kernel on a column-scaled case (d = 2,000,000), scaled by the units a full launch processes.
 NCU_TRAFFIC_BYTES = {
-    # profiles/sgp_step_tma_resnet50_small_ncu.md: 1479.6 MB per launch at d = 2,000,000, x (25,557,032 / 2,000,000)
+    # 1479.6 MB per launch at d = 2,000,000, x (25,557,032 / 2,000,000)
     "resnet50": 18.907e9,
-    # profiles/sgp_step_regs_osgp1_small_ncu.md: 1990.5 MB per launch at d = 2,000,000, same scaling
+    # 1990.5 MB per launch at d = 2,000,000, same scaling
     "resnet50_osgp1": 25.436e9,
 }
 

@@ -1,4 +1,4 @@
-"""Parity at the full BASELINE sizes, in the launch configuration the benchmark times.
+"""Parity at the full workload sizes, in the launch configuration the benchmark times.
 
 The float64 oracle cannot run 8e8 .. 6.4e9 elements in seconds, but every column of the SGP recursion
 evolves independently of every other column, so the oracle is run on sampled column windows (first

@@ -103,7 +103,7 @@ def _compare(w, out, K=None, write_z=True, P_of_k=None):
     return st
 
 
-# ------------------------------------------------------------------ the BASELINE configurations, oracle-sized
+# ------------------------------------------------------------------ the five workload configurations, oracle-sized
 def test_config1_tiny_closed_loop(binding, inputs):
     """n=8, d=4096, K=100, one-peer graph, Nesterov; g = z - c + noise computed from each side's OWN z."""
     from oracle import sgp as osgp
