@@ -504,3 +504,14 @@ def test_bounded_wait_reports_status_instead_of_hanging(binding, inputs):
         h.step(ref[0], ref[1], ref[2], G, ref[3], 0, w.lr, w.momentum, 0.0, True)
         torch.cuda.synchronize()
         assert torch.equal(X, ref[0]) and torch.equal(Z, ref[3]) and torch.equal(M, ref[2])
+
+
+@pytest.mark.parametrize("n,tau,nesterov", [(1, 2, True), (2, 1, True), (3, 3, False), (2, 1, False)])
+def test_degenerate_node_counts_with_delay(binding, inputs, n, tau, nesterov):
+    """n = 1 (no peers: the ring stays empty), n = 2 (one hop, the two nodes swap), heavy-ball with a ring."""
+    w = inputs.Workload("degenerate", n=n, d=777, K=9, graph="exp", peers=1, lr=0.1, momentum=0.9, nesterov=nesterov,
+                        tau=tau, weight_decay=1e-3)
+    out = _run_gpu(binding, inputs, w)
+    _compare(w, out)
+    if n == 1:
+        assert np.array_equal(out["W"], np.ones(1, dtype=np.float32)) and not out["ring"][0].any()
