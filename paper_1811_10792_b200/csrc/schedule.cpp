@@ -113,6 +113,20 @@ SgpStepCsr transpose_uniform(int n, const OutLists &out) {
   return s;
 }
 
+// True when all rows of P are equal: then x_i' = sum_j p_j h_j is the same vector for every receiver.
+bool rows_are_uniform(const SgpStepCsr &s, int n) {
+  const int32_t len = s.rowptr[1] - s.rowptr[0];
+  for (int i = 1; i < n; ++i) {
+    const int32_t b = s.rowptr[static_cast<size_t>(i)];
+    if (s.rowptr[static_cast<size_t>(i) + 1] - b != len) return false;
+    for (int32_t e = 0; e < len; ++e)
+      if (s.col[static_cast<size_t>(b + e)] != s.col[static_cast<size_t>(e)] ||
+          s.val[static_cast<size_t>(b + e)] != s.val[static_cast<size_t>(e)])
+        return false;
+  }
+  return true;
+}
+
 struct Edge {
   int32_t sender, receiver;
   float w;
@@ -208,6 +222,7 @@ int sgp_schedule_build(sgp_schedule **out, int n, const sgp_graph_desc *g) {
     delete s;
     return rc;
   }
+  for (SgpStepCsr &c : s->steps) c.uniform_rows = n > 1 && rows_are_uniform(c, n);
   *out = s;
   return SGP_OK;
 }

@@ -11,6 +11,7 @@ struct SgpStepCsr {
   std::vector<int32_t> col;     // senders, ascending inside each row
   std::vector<float> val;       // p_ij
   int32_t max_indeg = 0;
+  bool uniform_rows = false;    // every receiver has the same in-neighbour list and weights (e.g. the complete graph)
 };
 
 struct sgp_schedule {

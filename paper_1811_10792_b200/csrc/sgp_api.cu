@@ -201,6 +201,7 @@ void fill_params(const sgp_handle *h, const StepArgs &a, int64_t c0, int64_t c1,
   p.n = h->n;
   p.nnz = static_cast<int>(csr.col.size());
   p.update_w = update_w ? 1 : 0;
+  p.uniform_parts = 0;
   p.lr = a.lr;
   p.momentum = a.momentum;
   p.wd = a.wd;
@@ -294,12 +295,14 @@ int launch_regs(sgp_handle *h, const StepArgs &a, const Plan &pl, int64_t c0, in
   const size_t table_bytes = table_smem_bytes(h, p.nnz);
   if (h->const_ok[static_cast<size_t>(slot)]) p.table_mode = 0;
   else p.table_mode = table_bytes <= 40 * 1024 ? 1 : 2;
+  const bool uniform = h->tau == 0 && h->sched->slot(a.k).uniform_rows;
   // large n: one exchange tile (two barriers per tile) so that the row segments can stay twice as long
   p.single_buffer = h->opt_single_buffer == 1 ? 1 : (h->opt_single_buffer == 2 ? 0 : (auto_single_buffer(h->n) ? 1 : 0));
   size_t smem = 0;
   for (;;) {
+    p.uniform_parts = uniform ? static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(8, sgp::kThreads / tv))) : 0;
     smem = (p.single_buffer ? 1 : 2) * static_cast<size_t>(h->n) * tv * vec * 4 + 3 * static_cast<size_t>(h->n) * 4 +
-           (p.table_mode < 2 ? table_bytes : 0);
+           static_cast<size_t>(p.uniform_parts) * tv * vec * 4 + (p.table_mode < 2 ? table_bytes : 0);
     if (smem <= 110 * 1024 || tv <= min_tv) break;
     tv >>= 1;
   }
@@ -393,11 +396,13 @@ int launch_tma(sgp_handle *h, const StepArgs &a, const Plan &pl, int64_t c0, int
   const size_t table_bytes = table_smem_bytes(h, p.nnz);
   if (h->const_ok[static_cast<size_t>(slot)]) p.table_mode = 0;
   else p.table_mode = table_bytes <= 40 * 1024 ? 1 : 2;
-  const size_t fixed = 16 * sizeof(uint64_t) + 3 * static_cast<size_t>(h->n) * 4 + (p.table_mode < 2 ? table_bytes : 0);
+  const bool uniform = h->tau == 0 && h->sched->slot(a.k).uniform_rows;
+  size_t fixed = 16 * sizeof(uint64_t) + 3 * static_cast<size_t>(h->n) * 4 + (p.table_mode < 2 ? table_bytes : 0);
   const size_t budget = std::min<size_t>(static_cast<size_t>(h->smem_optin), (228 * 1024) / static_cast<size_t>(cps) - 2048);
   size_t smem = 0;
   for (;;) {
-    smem = static_cast<size_t>(stages) * arrays * h->n * tv * 16 + fixed;
+    p.uniform_parts = uniform ? static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(8, sgp::kTmaConsumers / tv))) : 0;
+    smem = static_cast<size_t>(stages) * arrays * h->n * tv * 16 + fixed + static_cast<size_t>(p.uniform_parts) * tv * 16;
     if (smem <= budget) break;
     if (h->opt_stages == 0 && stages > 2) --stages;
     else if (h->opt_tile_cols == 0 && tv > 8) tv >>= 1;

@@ -40,6 +40,8 @@ struct StepParams {
   int log2_tile_vecs;  // tile width in vectors (power of two)
   int update_w;        // 1: this launch also commits W (and the weight ring) for the step
   int table_mode;      // 0: copy table from the kernel argument, 1: copy from global, 2: read global in place
+  int uniform_parts;   // > 0: every row of P is the same (complete graph) and tau == 0: the mix is ONE weighted
+                       // column sum shared by all receivers, formed by this many interleaved partial sums
   int single_buffer;   // register kernel: 1 = one exchange tile and two barriers per tile (large n)
   int l2_hint;         // TMA kernel, L2 evict-first policy on the bulk copies: 0 none, 1 every array, 3 only G
                        // (dead after its read; X, M, V, ring are rewritten in place and keep the normal
@@ -215,7 +217,8 @@ sgp_step_regs_kernel(const __grid_constant__ StepParams p, const __grid_constant
   const int tile_items = n * tv;
   V *H0 = reinterpret_cast<V *>(smem_raw);
   V *H1 = p.single_buffer ? H0 : H0 + tile_items;
-  float *scratch = reinterpret_cast<float *>(H0 + (p.single_buffer ? 1 : 2) * tile_items);
+  V *partial = H0 + (p.single_buffer ? 1 : 2) * tile_items;          // uniform_parts x tv vectors (uniform rows only)
+  float *scratch = reinterpret_cast<float *>(partial + p.uniform_parts * tv);
   const CtaTables tab = cta_prologue<HAS_RING>(p, ct, scratch, kThreads);
 
   const int64_t ld = p.ld;
@@ -264,6 +267,33 @@ sgp_step_regs_kernel(const __grid_constant__ StepParams p, const __grid_constant
       }
     }
     __syncthreads();
+    // ---- phase 2, all receivers alike (complete graph): one weighted column sum, shared by every row
+    if (!HAS_RING && p.uniform_parts > 0) {
+      const int parts = p.uniform_parts;
+      const int e0 = tab.rowptr[0], e1 = tab.rowptr[1];
+      for (int idx = threadIdx.x; idx < tv * parts; idx += kThreads) {
+        const int c = idx & (tv - 1), part = idx >> p.log2_tile_vecs;
+        V acc = vzero<V>();
+        for (int e = e0 + part; e < e1; e += parts) acc = vfma(tab.val[e], H[(tab.col[e] << p.log2_tile_vecs) + c], acc);
+        partial[idx] = acc;
+      }
+      __syncthreads();
+      for (int item = threadIdx.x; item < tile_items; item += kThreads) {
+        const int row = item >> p.log2_tile_vecs;
+        const int c = item & (tv - 1);
+        const int64_t col = col0 + static_cast<int64_t>(c) * VEC;
+        if (col < p.col_end) {
+          const int64_t o = static_cast<int64_t>(row) * ld + col;
+          V acc = partial[c];
+          for (int part = 1; part < parts; ++part) acc = vadd(acc, partial[part * tv + c]);
+          st_stream(reinterpret_cast<V *>(p.X + o), acc);
+          if (HAS_Z) st_stream(reinterpret_cast<V *>(p.Z + o), vmul(tab.inv_w[row], acc));
+        }
+      }
+      buf ^= 1;
+      if (p.single_buffer) __syncthreads();
+      continue;
+    }
     // ---- phase 2: gather-mix over the step's in-neighbour lists, ring exchange, de-bias
     for (int base = 0; base < tile_items; base += kThreads * kItemsPerThread) {
       V ring_in[kItemsPerThread];
@@ -429,7 +459,8 @@ sgp_step_tma_kernel(const __grid_constant__ StepParams p, const __grid_constant_
   const size_t stage_bytes = static_cast<size_t>(kArrays) * tile_items * sizeof(float4);
   uint64_t *full_bar = reinterpret_cast<uint64_t *>(smem_raw + stages * stage_bytes);
   uint64_t *empty_bar = full_bar + kMaxStages;
-  float *scratch = reinterpret_cast<float *>(empty_bar + kMaxStages);
+  float4 *partial = reinterpret_cast<float4 *>(empty_bar + kMaxStages);   // uniform_parts x tv vectors
+  float *scratch = reinterpret_cast<float *>(partial + p.uniform_parts * tv);
   __shared__ int s_abort;
 
   const CtaTables tab = cta_prologue<HAS_RING>(p, ct, scratch, kTmaThreads);
@@ -545,6 +576,35 @@ sgp_step_tma_kernel(const __grid_constant__ StepParams p, const __grid_constant_
         }
       }
       consumer_barrier();
+      if (!HAS_RING && p.uniform_parts > 0) {
+        // all receivers alike (complete graph): one weighted column sum, shared by every row
+        const int parts = p.uniform_parts;
+        const int e0 = tab.rowptr[0], e1 = tab.rowptr[1];
+        for (int idx = ctid; idx < tv * parts; idx += kTmaConsumers) {
+          const int c = idx & (tv - 1), part = idx >> p.log2_tile_vecs;
+          float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+          for (int e = e0 + part; e < e1; e += parts) acc = vfma(tab.val[e], Xs[(tab.col[e] << p.log2_tile_vecs) + c], acc);
+          partial[idx] = acc;
+        }
+        consumer_barrier();
+        for (int item = ctid; item < tile_items; item += kTmaConsumers) {
+          const int row = item >> p.log2_tile_vecs;
+          const int c = item & (tv - 1);
+          const int64_t col = col0 + static_cast<int64_t>(c) * 4;
+          if (col < p.col_end) {
+            const int64_t o = static_cast<int64_t>(row) * ld + col;
+            float4 acc = partial[c];
+            for (int part = 1; part < parts; ++part) acc = vadd(acc, partial[part * tv + c]);
+            st_stream(reinterpret_cast<float4 *>(p.X + o), acc);
+            if (HAS_Z) st_stream(reinterpret_cast<float4 *>(p.Z + o), vmul(tab.inv_w[row], acc));
+          }
+        }
+        consumer_barrier();          // the partial sums are rewritten by the next tile
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty_bar + s);
+        continue;
+      }
       // phase 2: gather-mix, ring exchange, de-bias
       for (int item = ctid; item < tile_items; item += kTmaConsumers) {
         const int row = item >> p.log2_tile_vecs;

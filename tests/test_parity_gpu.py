@@ -515,3 +515,13 @@ def test_degenerate_node_counts_with_delay(binding, inputs, n, tau, nesterov):
     _compare(w, out)
     if n == 1:
         assert np.array_equal(out["W"], np.ones(1, dtype=np.float32)) and not out["ring"][0].any()
+
+
+@pytest.mark.parametrize("n,d", [(2, 1000), (7, 3000), (32, 8200), (64, 2052), (256, 1029)])
+@pytest.mark.parametrize("variant", [1, 3])
+def test_complete_graph_shared_column_sum_path(binding, inputs, n, d, variant):
+    """All receivers alike (complete graph): the mix is one column sum shared by every row; momentum and Z on."""
+    w = inputs.Workload("complete", n=n, d=d, K=6, graph="complete", lr=0.1, momentum=0.9, weight_decay=1e-4)
+    out = _run_gpu(binding, inputs, w, options={"variant": variant})
+    _compare(w, out)
+    assert np.abs(out["Z"] - out["Z"][0]).max() == 0.0               # every node holds the same vector, bit for bit
