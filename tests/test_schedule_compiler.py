@@ -192,3 +192,31 @@ def test_custom_random_weighted_schedules_bit_exact(binding, n, steps, seed):
         P = S.custom_mixing_matrix(n, send[sel], recv[sel], wt[sel].astype(np.float32))
         assert np.allclose(P.sum(axis=0), 1.0, atol=1e-6)
         _assert_slot_equal(sched, k, P)
+
+
+def test_header_is_valid_c_and_library_links_from_c(binding, tmp_path):
+    """A C99 program built with gcc against include/sgp.h and libsgp.so reproduces the oracle's schedule."""
+    import shutil
+    import subprocess
+    if shutil.which("gcc") is None:
+        pytest.skip("gcc not available")
+    exe = tmp_path / "c_abi_smoke"
+    lib_dir = os.path.dirname(binding.LIB_PATH)
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-I", os.path.join(ROOT, "include"),
+                    os.path.join(ROOT, "tests", "c_abi_smoke.c"), "-o", str(exe), "-L", lib_dir, "-l:libsgp.so",
+                    f"-Wl,-rpath,{lib_dir}"], check=True, capture_output=True, text=True)
+    n = 8
+    out = subprocess.run([str(exe), str(n)], check=True, capture_output=True, text=True).stdout.splitlines()
+    assert out[0].split() == ["version", str(binding.version()), "n", str(n), "period", "3"]
+    got = {}
+    for line in out[1:]:
+        k, i, j, p = line.split()
+        got[(int(k), int(i), int(j))] = float(p)
+    want = {}
+    for k in range(3):
+        P = S.mixing_matrix("exp", n, k, peers=1)
+        for i in range(n):
+            for j in range(n):
+                if P[i, j] != 0.0:
+                    want[(k, i, j)] = P[i, j]
+    assert got == want
