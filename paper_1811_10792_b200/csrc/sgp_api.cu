@@ -228,12 +228,23 @@ bool auto_single_buffer(int n) { return (n > 32 && n <= 64) || n > 128; }
 
 size_t table_smem_bytes(const sgp_handle *h, int nnz) { return (static_cast<size_t>(h->n) + 1 + 2 * static_cast<size_t>(nnz)) * 4; }
 
+// Tile width of the register-staged kernel (128-bit path): row segments of at least 1 KB and about 2048
+// vector items per tile, shrunk until the exchange tile(s) plus `fixed` bytes stay near 80 KB per CTA --
+// two resident CTAs then leave about half of the SM's 256 KB to the L1 that tracks the loads in flight
+// (measured: n = 48 at 2 x 100 KB reaches 0.74 of the copy bandwidth, at 2 x 50 KB 0.93).
+int64_t regs_tile_cols(const sgp_handle *h, size_t fixed) {
+  int64_t cols = std::max<int64_t>(256, int64_t{4} << floor_log2(std::max<int64_t>(1, 2048 / h->n)));
+  const size_t copies = auto_single_buffer(h->n) ? 1 : 2;
+  while (cols > 32 && copies * static_cast<size_t>(h->n) * cols * 4 + fixed > 80 * 1024) cols >>= 1;
+  return cols;
+}
+
 // Heuristics from measurements on B200.  The step is HBM-bound; what decides the achieved bandwidth
 // is the length of the contiguous row segments (>= 1 KB), the bytes in flight per SM and a grid that
 // is exactly one wave.  Measured (fraction of the copy bandwidth, rows on 1 KB boundaries):
 //   momentum, n <= 24 : register-staged 0.97, TMA 0.90      momentum, n = 32 : TMA 0.97, register-staged 0.95
 //   no momentum, n=16 : TMA 0.96, register-staged 0.87      tau = 1, n = 32  : register-staged 0.97
-// cps = 0 means "as many CTAs per SM as are resident" (asked of the occupancy calculator at launch).
+// cps = 0 means "as many CTAs per SM as are resident" (worked out at launch).
 // Explicit options override each field.
 Plan make_plan(const sgp_handle *h, int arrays, bool has_m, int nnz, bool vec) {
   Plan pl{1, 0, 2, 0};
@@ -247,24 +258,13 @@ Plan make_plan(const sgp_handle *h, int arrays, bool has_m, int nnz, bool vec) {
     } else if (has_m && per_kb >= 84 * 1024 && 2 * per_kb + fixed <= full_sm) {
       pl = Plan{3, 256, 2, 2 * per_kb + fixed <= half_sm ? 2 : 1};
     } else {
-      // register-staged: at least 1 KB row segments and about 2048 vector items per tile;
-      // the double-buffered exchange tile is 2 x n x tile_cols x 4 bytes
-      pl.tile_cols = std::max<int64_t>(256, int64_t{4} << floor_log2(std::max<int64_t>(1, 2048 / h->n)));
-      // keep the two resident CTAs' shared memory near half of the SM's 256 KB: the rest is the L1 that
-      // tracks the loads in flight (measured: n = 48 at 2 x 100 KB reaches 0.74, at 2 x 50 KB 0.93)
-      const size_t copies = auto_single_buffer(h->n) ? 1 : 2;
-      while (pl.tile_cols > 32 && copies * static_cast<size_t>(h->n) * pl.tile_cols * 4 + fixed > 80 * 1024) pl.tile_cols >>= 1;
+      pl.tile_cols = regs_tile_cols(h, fixed);
     }
   }
   if (h->opt_variant > 0 && (h->opt_variant == 1) != (pl.variant == 1)) {
     // the caller forces the other kernel family: take that family's defaults
     if (h->opt_variant == 1) {
-      pl = Plan{1, 256, 2, 0};
-      if (vec) {
-        pl.tile_cols = std::max<int64_t>(256, int64_t{4} << floor_log2(std::max<int64_t>(1, 2048 / h->n)));
-        const size_t copies = auto_single_buffer(h->n) ? 1 : 2;
-        while (pl.tile_cols > 32 && copies * static_cast<size_t>(h->n) * pl.tile_cols * 4 > 76 * 1024) pl.tile_cols >>= 1;
-      }
+      pl = Plan{1, vec ? regs_tile_cols(h, 4 * 1024) : 0, 2, 0};
     } else {
       pl = Plan{static_cast<int>(h->opt_variant), 256, 2, 2};
     }
@@ -283,7 +283,7 @@ int launch_regs(sgp_handle *h, const StepArgs &a, const Plan &pl, int64_t c0, in
   StepParams p{};
   fill_params(h, a, c0, c1, update_w, &p);
 
-  // tile width: about kThreads * kItemsPerThread items per tile, at least 128 bytes per row segment
+  // tile width: the plan's, else about four items per thread; at least 128 bytes per row segment
   const int64_t ncols = c1 - c0;
   const int min_tv = vec == 4 ? 8 : 32;
   int64_t tv = int64_t{1} << floor_log2(std::max<int64_t>(1, sgp::kThreads * 4 / h->n));
