@@ -407,7 +407,7 @@ def main():
                     "kernel": "sgp_step (fused update + mix + de-bias)", "algorithmic_bytes_per_launch": bpu * n * d,
                     "kernel_ms": kern_ms, "frac_of_nominal_8TBps": achieved / NOMINAL_HBM_GBS}
         cpu = None
-        if not args.no_cpu_baseline:
+        if not args.no_cpu_baseline and world == 1:          # the CPU oracle is timed in single-GPU runs only
             sample_cols = min(d, 1 << 20)
             dt, threads = oracle_sample_run(w, sample_cols, steps=8, warmup=1)
             cpu = {"value": n * sample_cols / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
