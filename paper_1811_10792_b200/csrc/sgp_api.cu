@@ -242,8 +242,8 @@ int64_t regs_tile_cols(const sgp_handle *h, size_t fixed) {
 // Heuristics from measurements on B200.  The step is HBM-bound; what decides the achieved bandwidth
 // is the length of the contiguous row segments (>= 1 KB), the bytes in flight per SM and a grid that
 // is exactly one wave.  Measured (fraction of the copy bandwidth, rows on 1 KB boundaries):
-//   momentum, n <= 24 : register-staged 0.97, TMA 0.90      momentum, n = 32 : TMA 0.97, register-staged 0.95
-//   no momentum, n=16 : TMA 0.96, register-staged 0.87      tau = 1, n = 32  : register-staged 0.97
+//   momentum, n <= 24 : register-staged 0.97, TMA 0.90      momentum, n = 32 : TMA 0.985, register-staged 0.95
+//   no momentum, n=16 : TMA 0.98, register-staged 0.97      tau = 1, n = 32  : register-staged 0.97
 // cps = 0 means "as many CTAs per SM as are resident" (worked out at launch).
 // Explicit options override each field.
 Plan make_plan(const sgp_handle *h, int arrays, bool has_m, int nnz, bool vec) {
@@ -253,7 +253,9 @@ Plan make_plan(const sgp_handle *h, int arrays, bool has_m, int nnz, bool vec) {
                          (table_smem_bytes(h, nnz) <= 40 * 1024 ? table_smem_bytes(h, nnz) : 0);
     const size_t per_kb = static_cast<size_t>(arrays) * h->n * 1024;   // one stage at 1 KB per row segment
     const size_t half_sm = 112 * 1024, full_sm = 224 * 1024;
-    if (!has_m && 2 * per_kb + fixed <= half_sm) {
+    if (!has_m && per_kb >= 24 * 1024 && per_kb <= 40 * 1024) {
+      // plain SGD with about 32 KB per stage (n = 16): two CTAs per SM, two stages: 0.98 against 0.97 for the
+      // register-staged kernel, which wins at every other n (n = 4: 0.97 against 0.93, n = 32: 0.98 against 0.88)
       pl = Plan{3, 256, 2, 2};
     } else if (has_m && per_kb >= 84 * 1024 && 2 * per_kb + fixed <= full_sm) {
       pl = Plan{3, 256, 2, 2 * per_kb + fixed <= half_sm ? 2 : 1};

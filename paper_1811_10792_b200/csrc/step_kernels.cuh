@@ -99,7 +99,8 @@ enum : int { kUpdSgd = 0, kUpdHeavyBall = 1, kUpdNesterov = 2, kUpdAdam = 3 };
 template <int UPD> struct UpdTraits {
   static constexpr bool kHasM = UPD != kUpdSgd;
   static constexpr bool kHasV = UPD == kUpdAdam;
-  static constexpr int kItems = UPD == kUpdAdam ? 3 : 4;   // items a thread of the register kernel keeps in flight
+  // items a thread of the register kernel keeps in flight: 12 to 16 vector loads with every optimiser
+  static constexpr int kItems = UPD == kUpdAdam ? 3 : (UPD == kUpdSgd ? 8 : 4);
 };
 
 // Local update of one element group: returns h = x^(k+1/2) and updates the optimiser state in place.
@@ -226,12 +227,17 @@ sgp_step_regs_kernel(const __grid_constant__ StepParams p, const __grid_constant
   const int64_t tile_cols = static_cast<int64_t>(tv) * VEC;
   const int64_t ntiles = (ncols + tile_cols - 1) / tile_cols;
   int buf = 0;
+  // The tile is worked off in batches of at most kItemsPerThread items per thread; the batches are made
+  // equal (e.g. 1280 items: 3 + 2 per thread, not 4 + 1) so that no batch runs with few loads in flight.
+  const int batches = (tile_items + kThreads * kItemsPerThread - 1) / (kThreads * kItemsPerThread);
+  const int q_max = ((tile_items + batches - 1) / batches + kThreads - 1) / kThreads;   // items per thread per batch
+  const int batch_items = q_max * kThreads;
 
   for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
     const int64_t col0 = p.col_begin + tile * tile_cols;
     V *H = buf ? H1 : H0;
     // ---- phase 1: local update, all batches of this tile
-    for (int base = 0; base < tile_items; base += kThreads * kItemsPerThread) {
+    for (int base = 0; base < tile_items; base += batch_items) {
       V x[kItemsPerThread], g[kItemsPerThread], u[kItemsPerThread], vv[kItemsPerThread];
       bool ok[kItemsPerThread];
       int64_t off[kItemsPerThread];
@@ -241,7 +247,7 @@ sgp_step_regs_kernel(const __grid_constant__ StepParams p, const __grid_constant
         const int row = item >> p.log2_tile_vecs;
         const int c = item & (tv - 1);
         const int64_t col = col0 + static_cast<int64_t>(c) * VEC;
-        ok[q] = (item < tile_items) && (col < p.col_end);
+        ok[q] = (q < q_max) && (item < tile_items) && (col < p.col_end);
         off[q] = static_cast<int64_t>(row) * ld + col;
       }
 #pragma unroll
@@ -261,7 +267,7 @@ sgp_step_regs_kernel(const __grid_constant__ StepParams p, const __grid_constant
           if (HAS_M) st_stream(reinterpret_cast<V *>(p.M + off[q]), u[q]);
           if (HAS_V) st_stream(reinterpret_cast<V *>(p.V + off[q]), vv[q]);
           H[item] = h;
-        } else if (item < tile_items) {
+        } else if (q < q_max && item < tile_items) {
           H[item] = vzero<V>();
         }
       }
@@ -295,7 +301,7 @@ sgp_step_regs_kernel(const __grid_constant__ StepParams p, const __grid_constant
       continue;
     }
     // ---- phase 2: gather-mix over the step's in-neighbour lists, ring exchange, de-bias
-    for (int base = 0; base < tile_items; base += kThreads * kItemsPerThread) {
+    for (int base = 0; base < tile_items; base += batch_items) {
       V ring_in[kItemsPerThread];
       if (HAS_RING) {
 #pragma unroll
@@ -304,7 +310,7 @@ sgp_step_regs_kernel(const __grid_constant__ StepParams p, const __grid_constant
           const int row = item >> p.log2_tile_vecs;
           const int c = item & (tv - 1);
           const int64_t col = col0 + static_cast<int64_t>(c) * VEC;
-          if (item < tile_items && col < p.col_end)
+          if (q < q_max && item < tile_items && col < p.col_end)
             ring_in[q] = ld_inplace(reinterpret_cast<const V *>(p.ring_x + static_cast<int64_t>(row) * ld + col));
         }
       }
@@ -314,7 +320,7 @@ sgp_step_regs_kernel(const __grid_constant__ StepParams p, const __grid_constant
         const int row = item >> p.log2_tile_vecs;
         const int c = item & (tv - 1);
         const int64_t col = col0 + static_cast<int64_t>(c) * VEC;
-        if (item < tile_items && col < p.col_end) {
+        if (q < q_max && item < tile_items && col < p.col_end) {
           const int64_t o = static_cast<int64_t>(row) * ld + col;
           V acc = vzero<V>(), offd = vzero<V>();
           const int e1 = tab.rowptr[row + 1];
