@@ -221,10 +221,10 @@ struct Plan {
   int cps;
 };
 
-// Register-staged kernel: one exchange tile (two barriers per tile) where that keeps the row segments at
-// 1 KB (32 < n <= 64: 0.95 against 0.92) or at 256 B (n > 128: 0.91 against 0.70); two tiles and one
-// barrier elsewhere (n = 128: 0.94 against 0.91).
-bool auto_single_buffer(int n) { return (n > 32 && n <= 64) || n > 128; }
+// Register-staged kernel: one exchange tile (two barriers per tile) where that keeps the row segments long
+// (n = 64: 1 KB segments 0.95 against 0.92; n = 80: 0.97 against 0.82; n = 96: 512 B 0.92 against 0.89;
+// n > 128: 256 B 0.91 against 0.70); two tiles and one barrier elsewhere (n = 112, 128: 0.94 against 0.92).
+bool auto_single_buffer(int n) { return (n > 32 && n <= 104) || n > 128; }
 
 size_t table_smem_bytes(const sgp_handle *h, int nnz) { return (static_cast<size_t>(h->n) + 1 + 2 * static_cast<size_t>(nnz)) * 4; }
 
@@ -235,7 +235,8 @@ size_t table_smem_bytes(const sgp_handle *h, int nnz) { return (static_cast<size
 int64_t regs_tile_cols(const sgp_handle *h, size_t fixed) {
   int64_t cols = std::max<int64_t>(256, int64_t{4} << floor_log2(std::max<int64_t>(1, 2048 / h->n)));
   const size_t copies = auto_single_buffer(h->n) ? 1 : 2;
-  while (cols > 32 && copies * static_cast<size_t>(h->n) * cols * 4 + fixed > 80 * 1024) cols >>= 1;
+  const size_t cap = (copies == 1 ? 88 : 80) * 1024;     // n = 80 at 85 KB: 0.97; n = 96 at 102 KB: 0.79
+  while (cols > 32 && copies * static_cast<size_t>(h->n) * cols * 4 + fixed > cap) cols >>= 1;
   return cols;
 }
 
