@@ -253,13 +253,16 @@ Plan make_plan(const sgp_handle *h, int arrays, bool has_m, int nnz, bool vec) {
     const size_t fixed = 16 * sizeof(uint64_t) + 3 * static_cast<size_t>(h->n) * 4 + 1024 +
                          (table_smem_bytes(h, nnz) <= 40 * 1024 ? table_smem_bytes(h, nnz) : 0);
     const size_t per_kb = static_cast<size_t>(arrays) * h->n * 1024;   // one stage at 1 KB per row segment
-    const size_t half_sm = 112 * 1024, full_sm = 224 * 1024;
+    const size_t full_sm = 224 * 1024;
     if (!has_m && per_kb >= 24 * 1024 && per_kb <= 40 * 1024) {
       // plain SGD with about 32 KB per stage (n = 16): two CTAs per SM, two stages: 0.98 against 0.97 for the
       // register-staged kernel, which wins at every other n (n = 4: 0.97 against 0.93, n = 32: 0.98 against 0.88)
       pl = Plan{3, 256, 2, 2};
-    } else if (has_m && per_kb >= 84 * 1024 && 2 * per_kb + fixed <= full_sm) {
-      pl = Plan{3, 256, 2, 2 * per_kb + fixed <= half_sm ? 2 : 1};
+    } else if (has_m && per_kb == 96 * 1024 && 2 * per_kb + fixed <= full_sm) {
+      // momentum with exactly 96 KB per stage (n = 32 with three arrays): one CTA per SM, two stages: 0.985 on
+      // the one-peer graph against 0.97 for the register-staged kernel; at n = 26..30, 34, 36 the
+      // register-staged kernel wins (0.96-0.99 against 0.91-0.95)
+      pl = Plan{3, 256, 2, 1};
     } else {
       pl.tile_cols = regs_tile_cols(h, fixed);
     }
