@@ -254,7 +254,13 @@ Plan make_plan(const sgp_handle *h, int arrays, bool has_m, int nnz, bool vec) {
                          (table_smem_bytes(h, nnz) <= 40 * 1024 ? table_smem_bytes(h, nnz) : 0);
     const size_t per_kb = static_cast<size_t>(arrays) * h->n * 1024;   // one stage at 1 KB per row segment
     const size_t full_sm = 224 * 1024;
-    if (!has_m && per_kb >= 24 * 1024 && per_kb <= 40 * 1024) {
+    // The pipelined kernel has ONE consumer group, so its gather is on the critical path: it is only used
+    // for sparse steps (at most three in-neighbours per node on average; with five it drops to 0.94, with
+    // nine to 0.88, while the register-staged kernel holds 0.98 and 0.95).
+    const bool sparse = static_cast<int64_t>(nnz) <= 3 * static_cast<int64_t>(h->n);
+    if (!sparse) {
+      pl.tile_cols = regs_tile_cols(h, fixed);
+    } else if (!has_m && per_kb >= 24 * 1024 && per_kb <= 40 * 1024) {
       // plain SGD with about 32 KB per stage (n = 16): two CTAs per SM, two stages: 0.98 against 0.97 for the
       // register-staged kernel, which wins at every other n (n = 4: 0.97 against 0.93, n = 32: 0.98 against 0.88)
       pl = Plan{3, 256, 2, 2};
