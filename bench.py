@@ -128,10 +128,15 @@ def oracle_sample_run(w, sample_cols: int, steps: int, warmup: int):
     Returns (seconds per step, BLAS threads)."""
     import numpy as np
     import torch
+    from oracle import schedule as osched
     from oracle import sgp as osgp
     from paper_1811_10792_b200 import inputs
-    sys.path.insert(0, os.path.join(ROOT, "tests"))
-    from parity_util import oracle_P_of_k
+
+    def oracle_P_of_k(w):
+        if w.graph == "random":
+            return lambda k: osched.mixing_matrix("random", w.n, k, seed=w.seed, max_outdeg=w.max_outdeg,
+                                                  num_steps=w.num_steps)
+        return lambda k: osched.mixing_matrix(w.graph, w.n, k, peers=w.peers)
 
     x0 = inputs.initial_x(w, device="cpu", d=sample_cols).numpy().astype(np.float64)
     G = torch.empty((w.n, sample_cols), dtype=torch.float32)
@@ -206,8 +211,6 @@ def run_sweep(args):
     """Scaling sweep (random digraphs, Nesterov, Z written): one JSON line per (n, d) point that fits 150 GB."""
     import torch
     from paper_1811_10792_b200 import binding, inputs
-    sys.path.insert(0, os.path.join(ROOT, "tests"))
-    from parity_util import graph_desc
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(dev)
     peak, peak_kind = measured_peak()
@@ -224,7 +227,7 @@ def run_sweep(args):
             inputs.gradient(w, 0, G)
             Wt = torch.ones(n, device=dev)
             K = w.K
-            with binding.Sgp(n, d, graph_desc(w, binding), ld=ld) as h:
+            with binding.Sgp(n, d, binding.graph_desc(w), ld=ld) as h:
                 for k in range(max(3, args.warmup)):
                     h.step(X, Wt, M, G, Z, k, w.lr, w.momentum, 0.0, True)
                 torch.cuda.synchronize()
@@ -300,8 +303,6 @@ def main():
     import torch
     import torch.distributed as dist
     from paper_1811_10792_b200 import binding     # raises if the CUDA library is missing: no fallback
-    sys.path.insert(0, os.path.join(ROOT, "tests"))
-    from parity_util import graph_desc
 
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device (there is no CPU path)")
@@ -336,7 +337,7 @@ def main():
         G = matrix()
         inputs.gradient(w, k, G)
         Gs.append(G)
-    h = binding.Sgp(n, d, graph_desc(w, binding), tau=w.tau, ld=ld)
+    h = binding.Sgp(n, d, binding.graph_desc(w), tau=w.tau, ld=ld)
     for kv in args.option:
         key, val = kv.split("=")
         h.set_option(key, int(val))

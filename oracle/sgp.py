@@ -15,15 +15,14 @@ Readings fixed here where the paper leaves a choice:
   * K steps means k = 0 .. K-1; u^(0) = 0; w^(0) = 1; z^(0) = x^(0).
   * Weight decay adds lambda * x (the biased numerator the optimiser steps on,
     App. C description of the compute thread) to the gradient.
-  * Adam: the paper combines SGP with "the Adam preconditioner" for its Transformer runs (Sec. 6.2,
-    App. C.1) without a listing.  Reading: the bias-corrected Adam step of Kingma & Ba replaces
+  * Adam: Sec. 6.2 / App. C.1 run Adam-preconditioned SGP on the Transformer without a listing.  Reading: the bias-corrected Adam step of Kingma & Ba replaces
     Alg. 3 lines 4-5 (gradient taken at z, step applied to the numerator x, both moment vectors local
     to a node and never gossiped); weight decay is added to the gradient as for SGD.
   * Delay tau: the self term p_ii h_i is never delayed; every other message
     (p_ij h_j, p_ij w_j) sent at step k is added at step k + tau, i.e. it lands
     in x^(k+tau+1); messages are sent every step; both parts accumulate;
-    virtual nodes start at zero.  For tau = 1 this is Alg. 2 ("always received
-    with 1 iteration of staleness", Table 4 caption).
+    virtual nodes start at zero.  For tau = 1 this is Alg. 2 (Table 4 caption:
+    fixed 1-step delay).
 
 Pins: tests/test_oracle_sgp.py.
 """

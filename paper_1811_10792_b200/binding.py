@@ -323,6 +323,17 @@ def step_static(n: int, d: int, ld: int, rowptr, col, val, X, W, M, G, Z, lr: fl
                                 _stream_ptr(stream)), "sgp_step_static")
 
 
+def graph_desc(w) -> GraphDesc:
+    """Schedule descriptor of a workload from `inputs` (marshalling of its graph fields, nothing else)."""
+    if w.graph == "exp":
+        return GraphDesc.exp_peers(w.peers)
+    if w.graph == "complete":
+        return GraphDesc.complete()
+    if w.graph == "random":
+        return GraphDesc.random_outdeg(w.seed, w.num_steps, w.max_outdeg)
+    raise ValueError(w.graph)
+
+
 def empty_matrix(n: int, d: int, device="cuda", pitch_multiple: int = 256, fill=None):
     """n x d float32 view whose rows start `ld` floats apart, ld = d rounded up to `pitch_multiple`.
 

@@ -104,8 +104,8 @@ template <int UPD> struct UpdTraits {
 };
 
 // Local update of one element group: returns h = x^(k+1/2) and updates the optimiser state in place.
-// SGD: Alg. 1 line 4.  Momentum / Nesterov: Alg. 3 lines 4-5.  Adam (Sec. 6.2, App. C.1: "combine SGP
-// with the Adam preconditioner"): bias-corrected Adam step on the numerator, moments stay local.
+// SGD: Alg. 1 line 4.  Momentum / Nesterov: Alg. 3 lines 4-5.  Adam (Sec. 6.2, App. C.1: Adam-preconditioned
+// SGP): bias-corrected Adam step on the numerator, moments stay local.
 // Weight decay adds wd * x to the gradient in every case.
 template <int UPD, typename V>
 __device__ __forceinline__ V local_update(V x, V g, V &u, V &v, const StepParams &p) {

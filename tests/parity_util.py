@@ -22,13 +22,7 @@ def oracle_P_of_k(w):
 
 
 def graph_desc(w, binding):
-    if w.graph == "exp":
-        return binding.GraphDesc.exp_peers(w.peers)
-    if w.graph == "complete":
-        return binding.GraphDesc.complete()
-    if w.graph == "random":
-        return binding.GraphDesc.random_outdeg(w.seed, w.num_steps, w.max_outdeg)
-    raise ValueError(w.graph)
+    return binding.graph_desc(w)
 
 
 def assert_close(name, got, want, tol=REL_TOL):

@@ -2,6 +2,8 @@
 on the same seeded inputs.  Sizes span several column tiles and a ragged tail; the w != 1 cases
 (irregular graphs, delayed messages) are included because regular graphs cannot detect a broken
 weight path."""
+from fractions import Fraction
+
 import numpy as np
 import pytest
 import torch
@@ -213,7 +215,7 @@ def test_complete_graph_is_parallel_sgd(binding, inputs):
 def test_custom_four_node_graph_weights_converge(binding, inputs):
     """The paper's worked 4-node matrix as a custom schedule: w -> (8,16,16,12)/13 and z -> average."""
     rows = read_golden("four_node_update_equations.txt")
-    recv = [int(r[0]) for r in rows]; send = [int(r[1]) for r in rows]; wt = [float(eval(r[2])) for r in rows]
+    recv = [int(r[0]) for r in rows]; send = [int(r[1]) for r in rows]; wt = [float(Fraction(r[2])) for r in rows]
     g = binding.GraphDesc.custom(1, [0] * len(rows), send, recv, wt)
     from oracle import schedule as osched
     P = osched.custom_mixing_matrix(4, send, recv, np.asarray(wt, dtype=np.float32))

@@ -4,6 +4,8 @@ import ctypes as C
 import os
 import re
 
+from fractions import Fraction
+
 import numpy as np
 import pytest
 
@@ -59,7 +61,7 @@ def _four_node_edges():
     rows = read_golden("four_node_update_equations.txt")
     recv = [int(r[0]) for r in rows]
     send = [int(r[1]) for r in rows]
-    wt = [float(eval(r[2])) for r in rows]     # "1/2", "1/3"
+    wt = [float(Fraction(r[2])) for r in rows]     # "1/2", "1/3"
     return send, recv, wt
 
 
