@@ -12,7 +12,8 @@ CUDA library's schedule compiler.
 
 Pins (tests/test_oracle_schedule.py): the worked 4-node matrix and its update
 equations, exact consensus after log2(n) one-peer steps, the averaging-quality
-figures quoted in App. A for n = 32, column-stochasticity of every kind.
+figures quoted in App. A for n = 32, column-stochasticity of every kind, the bipartite graph's perfect
+odd-even matching and symmetry.
 """
 from __future__ import annotations
 
@@ -57,6 +58,36 @@ def exp_out_neighbours(n: int, k: int, peers: int) -> list[list[int]]:
             s.add((i + hop) % n)
         out.append(sorted(s))
     return out
+
+
+def bipartite_exp_hops(n: int) -> list[int]:
+    """Hop distances of the undirected bipartite exponential graph (App. A, "Undirected exponential graph").
+
+    Odd-numbered nodes pair with the even-numbered nodes 2^1 - 1, 2^2 - 1, ..., 2^floor(log2(n-1)) - 1 hops
+    away.  Reading for n = 2, where that list is empty: the single hop 1 (the only even node there is).
+    """
+    if n < 2 or n % 2 != 0:
+        raise ValueError("the bipartite exponential graph needs an even number of nodes")
+    top = (n - 1).bit_length() - 1               # floor(log2(n-1))
+    return [(1 << j) - 1 for j in range(1, top + 1)] or [1]
+
+
+def bipartite_exp_out_neighbours(n: int, k: int) -> list[list[int]]:
+    """Out-neighbour sets (self included) of step k of the undirected bipartite exponential graph.
+
+    Odd node i sends to the even node (i + hop_k) mod n and that node sends back to i (App. A: the odd
+    node waits for the message in return), the hop cycling through `bipartite_exp_hops` one entry per
+    step like the one-peer directed schedule.  Every node therefore has exactly one partner per step
+    and the edge set is symmetric.
+    """
+    hops = bipartite_exp_hops(n)
+    hop = hops[k % len(hops)]
+    partner = [None] * n
+    for i in range(1, n, 2):                     # odd nodes initiate
+        j = (i + hop) % n
+        partner[i] = j
+        partner[j] = i
+    return [sorted({i, partner[i]}) for i in range(n)]
 
 
 def complete_out_neighbours(n: int) -> list[list[int]]:
@@ -133,12 +164,15 @@ def mixing_matrix(kind: str, n: int, k: int, *, peers: int = 1, seed: int = 0,
     """P^(k) for the named schedule.
 
     ``exp``: c-peer directed exponential graph; ``complete``: all-to-all;
+    ``bipartite``: undirected bipartite exponential graph (symmetric pairs);
     ``random``: the hashed random digraph, repeating with period ``num_steps``.
     """
     if kind == "exp":
         return uniform_mixing_matrix(exp_out_neighbours(n, k, peers))
     if kind == "complete":
         return uniform_mixing_matrix(complete_out_neighbours(n))
+    if kind == "bipartite":
+        return uniform_mixing_matrix(bipartite_exp_out_neighbours(n, k))
     if kind == "random":
         kk = k % num_steps if num_steps > 0 else k
         return uniform_mixing_matrix(random_out_neighbours(n, kk, seed, max_outdeg))
@@ -150,6 +184,8 @@ def schedule_period(kind: str, n: int, *, peers: int = 1, num_steps: int = 0) ->
         return max(1, exp_cycle_length(n))
     if kind == "complete":
         return 1
+    if kind == "bipartite":
+        return len(bipartite_exp_hops(n))
     if kind == "random":
         return num_steps
     raise ValueError(kind)

@@ -23,6 +23,14 @@ Readings fixed here where the paper leaves a choice:
     in x^(k+tau+1); messages are sent every step; both parts accumulate;
     virtual nodes start at zero.  For tau = 1 this is Alg. 2 (Table 4 caption:
     fixed 1-step delay).
+  * send_period s (Alg. 2 line 5 taken literally with s = tau; Sec. 3: nodes send every tau
+    iterations): a node sends only on steps with k mod s = 0; on every other step it keeps its
+    whole half step (Alg. 2 lines 10-11: the step's mixing matrix is the identity), while messages
+    sent earlier still arrive tau steps after they were sent.  The c-th transmission uses the
+    c-th matrix of the schedule, P^(k/s) (App. A describes the peer cycle per transmission).
+    s = 1 is the reading above.
+  * biased (Sec. 6.1 / Table 4, "biased 1-OSGP": the push-sum weight is not used): z = x; the
+    weights are still mixed so that they can be inspected, they just do not enter z.
 
 Pins: tests/test_oracle_sgp.py.
 """
@@ -41,6 +49,7 @@ class SGPState:
     u: np.ndarray                      # n x d momentum buffers
     z: np.ndarray                      # n x d de-biased parameters
     v: np.ndarray = None               # n x d Adam second moments (u holds the first moments)
+    h: np.ndarray = None               # n x d half step x^(k+1/2) of the latest iteration (before the mix)
     transit_x: deque = field(default_factory=deque)   # tau in-flight (n x d) messages, oldest first
     transit_w: deque = field(default_factory=deque)   # tau in-flight (n) weight messages
 
@@ -116,40 +125,53 @@ def mix_delayed(P, h, w, transit_x, transit_w):
     return x_next, w_next
 
 
-def sgp_step(st: SGPState, g, P, lr, momentum=0.0, nesterov=True, weight_decay=0.0, adam=None) -> SGPState:
+def sgp_step(st: SGPState, g, P, lr, momentum=0.0, nesterov=True, weight_decay=0.0, adam=None,
+             biased=False) -> SGPState:
     """One full SGP iteration in place on ``st`` (gradient g was taken at st.z).
 
-    ``adam`` = (t, beta1, beta2, eps) switches the local update to Adam.
+    ``adam`` = (t, beta1, beta2, eps) switches the local update to Adam.  ``biased`` leaves the
+    push-sum weight out of z (Table 4, biased 1-OSGP).  The half step is kept in ``st.h``.
     """
     if adam is None:
         h, st.u = local_update(st.x, st.u, g, lr, momentum, nesterov, weight_decay)
     else:
         t, beta1, beta2, eps = adam
         h, st.u, st.v = local_update_adam(st.x, st.u, st.v, g, t, lr, beta1, beta2, eps, weight_decay)
+    st.h = h
     if len(st.transit_x) == 0:
         st.x, st.w = mix(P, h, st.w)
     else:
         st.x, st.w = mix_delayed(P, h, st.w, st.transit_x, st.transit_w)
-    st.z = st.x / st.w[:, None]                        # Alg. 1 line 8
+    if biased:
+        st.z = st.x.copy()                             # Table 4, biased 1-OSGP: w ignored
+    else:
+        st.z = st.x / st.w[:, None]                    # Alg. 1 line 8
     return st
 
 
 def sgp_run(x0, K, P_of_k, grad_of_k, lr, momentum=0.0, nesterov=True, weight_decay=0.0,
-            tau=0, history=None, adam=None) -> SGPState:
+            tau=0, history=None, adam=None, send_period=1, biased=False, half_steps=None) -> SGPState:
     """K iterations k = 0 .. K-1.
 
     ``P_of_k(k)`` returns the dense mixing matrix of step k; ``grad_of_k(k, z)``
     returns the n x d stochastic gradients evaluated at the de-biased ``z``.
     If ``history`` is a list, a snapshot (x, w, u, z) is appended after every step.
     ``adam`` = (beta1, beta2, eps) runs Adam-SGP (step count t = k + 1).
+    ``send_period`` = s: nodes transmit on steps k = 0, s, 2s, ... with the matrix P_of_k(k // s) and keep
+    everything (identity matrix) on the other steps (Alg. 2 lines 5-12).  If ``half_steps`` is a list the
+    half step x^(k+1/2) of every iteration is appended to it.
     """
     st = init_state(x0, tau)
+    n = st.x.shape[0]
     for k in range(K):
         g = grad_of_k(k, st.z)
-        sgp_step(st, g, P_of_k(k), lr, momentum, nesterov, weight_decay,
-                 adam=None if adam is None else (k + 1, *adam))
+        P = P_of_k(k // send_period) if k % send_period == 0 else np.eye(n)
+        sgp_step(st, g, P, lr, momentum, nesterov, weight_decay,
+                 adam=None if adam is None else (k + 1, *adam), biased=biased)
         if history is not None:
             history.append((st.x.copy(), st.w.copy(), st.u.copy(), st.z.copy()))
+        if half_steps is not None:
+            half_steps.append(st.h.copy())
     return st
 
 
@@ -166,6 +188,17 @@ def total_mass(st: SGPState):
         sx = sx + mx.sum(axis=0)
         sw = sw + mw.sum()
     return sx, sw
+
+
+def consensus_distance(st: SGPState):
+    """|| xbar - z_i ||_2 for every node, xbar = (1/n) * (sum of x over real AND virtual nodes).
+
+    The quantity bounded by the consensus lemma of the supplementary material; the node-wise average
+    counts the parameters that are in transit (definition of xbar after Eq. 4).
+    """
+    sx, _ = total_mass(st)
+    xbar = sx / st.x.shape[0]
+    return np.linalg.norm(st.z - xbar[None, :], axis=1)
 
 
 def param_deviation(a):

@@ -197,3 +197,53 @@ def test_fp32_weight_rounding_is_single_rounding_safe():
     # as a float32 division for every out-degree that can occur (n <= 256 and beyond)
     for length in range(1, 1025):
         assert np.float32(1.0 / length) == np.float32(1.0) / np.float32(length)
+
+
+# ---------------------------------------------------------------- App. A, undirected bipartite exponential graph
+def test_bipartite_hop_list_matches_formula_in_paper():
+    for row in read_golden("bipartite_exp_hops.txt"):
+        n, hops = int(row[0]), [int(t) for t in row[1:]]
+        assert S.bipartite_exp_hops(n) == hops
+        assert S.schedule_period("bipartite", n) == len(hops)
+    assert S.bipartite_exp_hops(2) == [1]
+    with pytest.raises(ValueError):
+        S.bipartite_exp_hops(7)
+
+
+@pytest.mark.parametrize("n", [2, 4, 8, 16, 32, 6, 10, 12])
+def test_bipartite_steps_are_perfect_odd_even_matchings(n):
+    for k in range(2 * S.schedule_period("bipartite", n)):
+        out = S.bipartite_exp_out_neighbours(n, k)
+        P = S.mixing_matrix("bipartite", n, k)
+        assert np.array_equal(P, P.T)                                    # undirected: message and reply
+        assert np.allclose(P.sum(axis=0), 1.0, atol=0) and np.allclose(P.sum(axis=1), 1.0, atol=0)
+        assert set(np.unique(P)) <= {0.0, 0.5}                           # self 1/2, partner 1/2 (App. C weights)
+        hop = S.bipartite_exp_hops(n)[k % S.schedule_period("bipartite", n)]
+        for i in range(n):
+            assert len(out[i]) == 2 and i in out[i]                      # exactly one partner each: regular graph
+            partner = [j for j in out[i] if j != i][0]
+            assert partner % 2 != i % 2                                  # bipartite: odd talks to even
+            if i % 2 == 1:
+                assert partner == (i + hop) % n                          # odd nodes initiate, hop taken forwards
+
+
+def test_bipartite_node1_partners_n8():
+    # hops 1 and 3: node 1 pairs with node 2, then node 4; node 0 is reached by node 7 (hop 1) and node 5 (hop 3)
+    assert S.bipartite_exp_out_neighbours(8, 0)[1] == [1, 2]
+    assert S.bipartite_exp_out_neighbours(8, 1)[1] == [1, 4]
+    assert S.bipartite_exp_out_neighbours(8, 0)[0] == [0, 7]
+    assert S.bipartite_exp_out_neighbours(8, 1)[0] == [0, 5]
+
+
+@pytest.mark.parametrize("n", [4, 8, 16, 32])
+def test_bipartite_cycle_contracts_towards_the_average(n):
+    # symmetric doubly stochastic steps keep the average and, over a few cycles, shrink every deviation from it
+    L = S.schedule_period("bipartite", n)
+    M = np.eye(n)
+    for k in range(8 * L):
+        M = S.mixing_matrix("bipartite", n, k) @ M
+    assert np.allclose(M.sum(axis=0), 1.0) and np.allclose(M.sum(axis=1), 1.0)
+    if n > 4:                                   # n = 4 has the single hop 1: two disjoint pairs never mix
+        assert _sigma2_sq(M) < 1e-2
+    else:
+        assert abs(_sigma2_sq(M) - 1.0) < 1e-12

@@ -318,3 +318,145 @@ def test_param_deviation_closed_forms():
     y = np.tile(x[0], (6, 1)); y[2] += e
     want = np.full(6, np.linalg.norm(e) / 6); want[2] *= 5
     assert np.allclose(O.param_deviation(y), want, rtol=1e-12)
+
+
+# ---------------------------------------------------------------- Alg. 2 line 5 taken literally: send every s steps
+@pytest.mark.parametrize("tau", [0, 1, 2, 3])
+def test_send_period_one_is_the_fixed_delay_reading(tau):
+    n, d, K = 8, 4, 9
+    rng = np.random.default_rng(70 + tau)
+    x0 = rng.standard_normal((n, d))
+    _, gfun = _rand_grads(n, d, K, 71)
+    Pk = lambda k: S.mixing_matrix("exp", n, k, peers=1)
+    a = O.sgp_run(x0, K, Pk, gfun, 0.05, momentum=0.9, tau=tau)
+    b = O.sgp_run(x0, K, Pk, gfun, 0.05, momentum=0.9, tau=tau, send_period=1)
+    for f in ("x", "w", "u", "z"):
+        assert np.array_equal(getattr(a, f), getattr(b, f))
+
+
+def test_send_period_weight_sequence_by_hand():
+    # n = 2, one-peer graph, tau = 2, transmissions on even steps only (Alg. 2 with send period tau).
+    # w after steps 0..5: 1/2 (kept half, nothing arrives), 1/2 (no send, nothing arrives), 1/4 + 1/2 = 3/4
+    # (the step-0 message lands), 3/4, 3/8 + 1/4 = 5/8 (the step-2 message was half of 1/2), 5/8: the 1-OSGP
+    # sequence 1/2, 3/4, 5/8, ... with every entry held for two steps.
+    hist = []
+    O.sgp_run(np.ones((2, 1)), 8, lambda k: S.mixing_matrix("exp", 2, k, peers=1), lambda k, z: np.zeros_like(z),
+              lr=0.1, tau=2, send_period=2, history=hist)
+    got = [h[1][0] for h in hist]
+    assert got == [0.5, 0.5, 0.75, 0.75, 0.625, 0.625, 0.6875, 0.6875]
+    assert all(np.allclose(h[3], 1.0, rtol=1e-15) for h in hist)       # z keeps the average throughout
+
+
+@pytest.mark.parametrize("tau,s", [(0, 2), (0, 3), (2, 2), (3, 3), (1, 2), (3, 2)])
+def test_send_period_conserves_mass_and_idles_between_transmissions(tau, s):
+    n, d, K = 8, 3, 13
+    rng = np.random.default_rng(80)
+    x0 = rng.standard_normal((n, d))
+    G, gfun = _rand_grads(n, d, K, 81)
+    lr = 0.1
+    used = []
+
+    def Pk(c):
+        used.append(c)
+        return S.mixing_matrix("exp", n, c, peers=1)
+
+    st = O.init_state(x0, tau)
+    for k in range(K):
+        x_before, transit_arriving = st.x.copy(), (st.transit_x[0].copy() if tau else 0.0)
+        mass_before, w_before = O.total_mass(st)
+        P = Pk(k // s) if k % s == 0 else np.eye(n)
+        O.sgp_step(st, G[k], P, lr)
+        mass_after, w_after = O.total_mass(st)
+        assert np.allclose(mass_after, mass_before - lr * G[k].sum(axis=0), rtol=0, atol=1e-13)
+        assert abs(w_after - n) < 1e-13
+        if k % s != 0:      # a node that does not transmit keeps its whole half step (Alg. 2 lines 10-11)
+            assert np.array_equal(st.x, (x_before - lr * G[k]) + transit_arriving)
+    # sgp_run hands the c-th transmission the c-th matrix of the schedule
+    calls = []
+    O.sgp_run(x0, K, lambda c: (calls.append(c), S.mixing_matrix("exp", n, c, peers=1))[1], gfun, lr, tau=tau,
+              send_period=s)
+    assert calls == list(range((K + s - 1) // s))
+
+
+# ---------------------------------------------------------------- Table 4: biased 1-OSGP (push-sum weight not used)
+def test_biased_osgp_closed_form():
+    # identical constant rows c, zero gradients, one-peer graph, tau = 1: the numerators shrink with the weights,
+    # x_i^(k) = c * w^(k) with w = 1/2, 3/4, 5/8, ... -> 2/3.  The de-biased z stays c; the biased one is x.
+    n, c = 8, np.array([3.0, -1.5, 0.25])
+    x0 = np.tile(c, (n, 1))
+    hist_b, hist_u = [], []
+    kw = dict(lr=0.1, tau=1)
+    O.sgp_run(x0, 40, lambda k: S.mixing_matrix("exp", n, k, peers=1), lambda k, z: np.zeros_like(z), biased=True,
+              history=hist_b, **kw)
+    O.sgp_run(x0, 40, lambda k: S.mixing_matrix("exp", n, k, peers=1), lambda k, z: np.zeros_like(z),
+              history=hist_u, **kw)
+    for k, wk in enumerate([0.5, 0.75, 0.625]):
+        assert np.allclose(hist_b[k][3], wk * x0, rtol=1e-15)
+        assert np.array_equal(hist_b[k][3], hist_b[k][0])               # z is the numerator itself
+        assert np.allclose(hist_u[k][3], x0, rtol=1e-15)
+        assert np.array_equal(hist_b[k][1], hist_u[k][1])               # the weights themselves are mixed as usual
+    assert np.allclose(hist_b[-1][3], (2.0 / 3.0) * x0, rtol=1e-9)
+
+
+def test_biased_flag_is_invisible_without_delay_on_regular_graphs():
+    n, d, K = 8, 3, 6
+    rng = np.random.default_rng(90)
+    x0 = rng.standard_normal((n, d))
+    _, gfun = _rand_grads(n, d, K, 91)
+    Pk = lambda k: S.mixing_matrix("exp", n, k, peers=2)
+    a = O.sgp_run(x0, K, Pk, gfun, 0.1, momentum=0.9)
+    b = O.sgp_run(x0, K, Pk, gfun, 0.1, momentum=0.9, biased=True)
+    assert np.allclose(a.z, b.z, rtol=1e-14, atol=1e-14)                 # w == 1: nothing to ignore
+
+
+# ---------------------------------------------------------------- half step accessor and consensus distance
+def test_half_step_accessor_closed_form():
+    # plain SGD: the half step is x - lr g whatever the graph; the mix is applied to exactly that
+    n, d = 4, 5
+    rng = np.random.default_rng(100)
+    x0 = rng.standard_normal((n, d))
+    G, gfun = _rand_grads(n, d, 3, 101)
+    halves, hist = [], []
+    P = lambda k: S.mixing_matrix("exp", n, k, peers=1)
+    O.sgp_run(x0, 3, P, gfun, 0.25, half_steps=halves, history=hist)
+    assert np.array_equal(halves[0], x0 - 0.25 * G[0])
+    for k in range(3):
+        assert np.allclose(hist[k][0], P(k) @ halves[k], rtol=1e-15, atol=1e-15)
+    # two nodes at a and b after the gradient step: each is ||a - b|| / 2 from their mean (Fig. 2 metric)
+    a, b = np.array([1.0, 2.0, 2.0]), np.array([-2.0, -2.0, 2.0])
+    halves = []
+    O.sgp_run(np.stack([a, b]), 1, lambda k: S.mixing_matrix("complete", 2, k), lambda k, z: np.zeros_like(z), 0.1,
+              half_steps=halves)
+    assert np.allclose(O.param_deviation(halves[0]), [2.5, 2.5])
+
+
+def test_consensus_distance_counts_mass_in_transit():
+    # n = 2, one-peer graph, tau = 1, zero gradients, rows a and b.  After one step x = (a/2, b/2), the messages
+    # (b/2, a/2) are in transit, w = 1/2 so z = (a, b).  xbar counts the transit: (a + b)/2, so both nodes are
+    # |a - b|/2 away; leaving the transit out would give xbar = (a + b)/4 instead.
+    a, b = np.array([4.0, 0.0]), np.array([0.0, 3.0])
+    st = O.sgp_run(np.stack([a, b]), 1, lambda k: S.mixing_matrix("exp", 2, k, peers=1),
+                   lambda k, z: np.zeros_like(z), 0.1, tau=1)
+    assert np.allclose(st.z, np.stack([a, b]))
+    assert np.allclose(O.consensus_distance(st), [2.5, 2.5])
+    # complete graph, no delay: every z is the average, distance 0
+    st = O.sgp_run(np.stack([a, b]), 1, lambda k: S.mixing_matrix("complete", 2, k), lambda k, z: np.zeros_like(z), 0.1)
+    assert np.all(O.consensus_distance(st) < 1e-15)
+    # asymmetric 4-node graph: distances shrink geometrically towards zero (consensus lemma)
+    P = np.array([[1/2, 0, 0, 1/3], [1/2, 1/2, 0, 1/3], [0, 1/2, 1/2, 0], [0, 0, 1/2, 1/3]])
+    x0 = np.random.default_rng(110).standard_normal((4, 6))
+    d10 = O.consensus_distance(O.sgp_run(x0, 10, lambda k: P, lambda k, z: np.zeros_like(z), 0.1))
+    d40 = O.consensus_distance(O.sgp_run(x0, 40, lambda k: P, lambda k, z: np.zeros_like(z), 0.1))
+    assert d40.max() < 1e-3 * d10.max()
+
+
+def test_bipartite_graph_keeps_unit_weights_d_psgd_case():
+    # symmetric doubly stochastic mixing (the D-PSGD topology of App. A): w == 1 at every step, z == x
+    n, d, K = 8, 4, 7
+    rng = np.random.default_rng(120)
+    x0 = rng.standard_normal((n, d))
+    _, gfun = _rand_grads(n, d, K, 121)
+    hist = []
+    O.sgp_run(x0, K, lambda k: S.mixing_matrix("bipartite", n, k), gfun, 0.1, momentum=0.9, history=hist)
+    for x, w, u, z in hist:
+        assert np.array_equal(w, np.ones(n)) and np.array_equal(z, x)
