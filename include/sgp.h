@@ -37,6 +37,18 @@ extern "C" {
 #define SGP_ERR_STATE    -5   /* call not valid for this handle (ring export with tau = 0; the current
                                  CUDA device is not the one the handle was created on)               */
 #define SGP_ERR_DEVICE   -6   /* a kernel reported a bounded wait that ran out (status word non-zero) */
+#define SGP_ERR_ZERO_WEIGHT -7 /* a push-sum weight is <= 0 or not a number: z = x / w is undefined      */
+#define SGP_ERR_INVARIANT -8  /* sgp_check: non-finite state, sum of weights != n, or a column sum drifted */
+
+/* Bits of the device status word (sgp_device_status).  Kernels only ever OR bits in; sgp_reset clears it. */
+#define SGP_STATUS_WAIT_TILE     1u   /* pipelined kernel: consumers gave up waiting for a tile              */
+#define SGP_STATUS_WAIT_STAGE    2u   /* pipelined kernel: the producer gave up waiting for a free stage     */
+#define SGP_STATUS_WAIT_DRAIN    4u   /* pipelined kernel: copies were still pending at exit                 */
+#define SGP_STATUS_ZERO_WEIGHT   8u   /* a weight was <= 0 or NaN (that node's z was written as 0, never inf) */
+#define SGP_STATUS_NONFINITE    16u   /* invariant check: non-finite entries in X or in the delay ring       */
+#define SGP_STATUS_WEIGHT_SUM   32u   /* invariant check: sum of weights incl. in transit differs from n     */
+#define SGP_STATUS_COLUMN_SUM   64u   /* invariant check: a column sum drifted from its reference            */
+#define SGP_STATUS_BOUNDS      128u   /* bounds-checked build only: an index was out of range, access skipped */
 
 #define SGP_MAX_NODES 256     /* n <= 256: one CTA keeps all n rows of a column tile on chip          */
 
@@ -45,7 +57,8 @@ typedef enum sgp_graph_kind {
   SGP_GRAPH_EXP_PEERS     = 0, /* App. A directed exponential graph, `peers` out-neighbours per step */
   SGP_GRAPH_COMPLETE      = 1, /* every entry 1/n (Sec. 3: equivalent to AllReduce parallel SGD)     */
   SGP_GRAPH_RANDOM_OUTDEG = 2, /* hashed random digraph, out-degree ~ U{1..min(max_outdeg, n-1)}     */
-  SGP_GRAPH_CUSTOM        = 3  /* explicit edge list with per-edge weights                           */
+  SGP_GRAPH_CUSTOM        = 3, /* explicit edge list with per-edge weights                           */
+  SGP_GRAPH_BIPARTITE_EXP = 4  /* App. A undirected bipartite exponential graph (the D-PSGD topology)   */
 } sgp_graph_kind;
 
 /*
@@ -54,6 +67,9 @@ typedef enum sgp_graph_kind {
  *              L = floor(log2(n-1)) + 1 hop distances (App. A); weights 1/|N_out| incl. self (App. C).
  *  RANDOM    : `num_steps` distinct steps, then the schedule repeats; draws are a keyed integer
  *              hash of (seed, step, node, draw) so that independent implementations agree bit for bit.
+ *  BIPARTITE : n even (SGP_ERR_ARG otherwise).  At step k odd node i and even node (i + hop_k) mod n exchange
+ *              messages, hop_k cycling through 2^1 - 1, ..., 2^floor(log2(n-1)) - 1 (n = 2: hop 1); weights 1/2
+ *              and 1/2, so P is symmetric doubly stochastic and the push-sum weights stay 1 (Sec. 4, App. A).
  *  CUSTOM    : num_edges quadruples (edge_step, edge_sender, edge_receiver, edge_weight); self-loops are
  *              listed explicitly; steps 0..num_steps-1, repeating.  Rejected with SGP_ERR_GRAPH if an
  *              index is out of range, an edge is duplicated, a weight is not finite and > 0, a
@@ -98,7 +114,9 @@ int sgp_schedule_get(const sgp_schedule *s, int64_t k, int32_t *rowptr, int32_t 
  * ------------------------------------------------------------------------------------------- */
 typedef struct sgp_handle sgp_handle;
 
-#define SGP_FLAG_NONE 0u
+#define SGP_FLAG_NONE   0u
+#define SGP_FLAG_BIASED 1u    /* Sec. 6.1 / Table 4 "biased OSGP" ablation: z = x, the push-sum weight is mixed and
+                                 kept in W but left out of the de-bias */
 
 /*
  * sgp_create: n nodes (1..SGP_MAX_NODES), d parameters per node, ld >= d the row pitch in floats of
@@ -172,11 +190,13 @@ int sgp_debias(sgp_handle *h, const float *d_X, const float *d_W, float *d_Z, vo
  * resident on the device; d_G and d_Z are device staging arrays of n x ld floats supplied by the
  * caller.  The columns are cut into chunks; chunk c's host->device copy, its fused step and its
  * device->host copy overlap with the neighbouring chunks on the handle's three internal streams.
- * Returns after everything has completed (synchronises).  chunk_cols <= 0 picks a default.
+ * Work the caller already enqueued on `stream` is waited for on the device (an event, no host
+ * synchronisation on entry).  Returns after everything has completed (synchronises the internal streams).
+ * chunk_cols <= 0 picks a default.
  */
 int sgp_step_host(sgp_handle *h, float *d_X, float *d_W, float *d_M, const float *h_G, float *h_Z,
                   float *d_G, float *d_Z, int64_t k, float lr, float momentum, float weight_decay,
-                  int nesterov, int64_t chunk_cols);
+                  int nesterov, int64_t chunk_cols, void *stream);
 
 /* Zeroes the delay ring (messages in transit are dropped: use only to restart a run). */
 int sgp_reset(sgp_handle *h, void *stream);
@@ -186,11 +206,47 @@ int sgp_ring_export(sgp_handle *h, float *d_ring_x, float *d_ring_w, void *strea
 int sgp_ring_import(sgp_handle *h, const float *d_ring_x, const float *d_ring_w, void *stream);
 
 /*
- * sgp_check: invariants of column-stochastic mixing (Sec. 2; delay model: mass in transit counts).
- * Writes to HOST h_stats[4]: { sum_i W_i + sum of ring weights (should equal n), min_i W_i,
- * number of non-finite entries of X, sum over all entries of X and the ring }.  Synchronises.
+ * sgp_colsum: per-column sums in fp64, d_out[c] = sum_i A[i, c] for the n x ld device array A (X, G, M, ...),
+ * plus, if include_ring != 0, every entry of the handle's delay ring in that column (the messages in transit:
+ * the virtual nodes of the delay model).  d_out is d doubles of DEVICE memory.  Asynchronous on `stream`.
+ * Column-stochastic mixing (Sec. 2: every column of P sums to one) conserves exactly these sums, so a caller can
+ * form the expected sums of the next state from sums of the current arrays -- e.g. for momentum SGD
+ *     colsum(X') + ring' = colsum(X) + ring - lr * (momentum * colsum(M') + colsum(G) + wd * colsum(X))   (Nesterov)
+ * -- and hand them to sgp_check.
  */
-int sgp_check(sgp_handle *h, const float *d_X, const float *d_W, double *h_stats, void *stream);
+int sgp_colsum(sgp_handle *h, const float *d_A, int include_ring, double *d_out, void *stream);
+
+/*
+ * sgp_check: invariants of column-stochastic mixing (Sec. 2; delay model: mass in transit counts).
+ * One pass over X and the ring; one thread per column, fp64 accumulation, warp-shuffle reductions.
+ * d_colsum_ref (DEVICE, d doubles, may be NULL): the expected per-column sums of X plus ring (see sgp_colsum).
+ * Writes to HOST h_stats[8]:
+ *   [0] sum_i W_i + sum of the ring weights (should equal n)      [1] min_i W_i (NaN reported as -1)
+ *   [2] number of non-finite entries of X and the ring            [3] sum over all entries of X and the ring
+ *   [4] max_c |colsum_c - ref_c|                                  [5] max_c |colsum_c - ref_c| / max(sum_i |x_ic|, |ref_c|)
+ *   [6] | [0] - n |                                               [7] the device status word after the check
+ * ([4], [5] are 0 without a reference).  The check ORs SGP_STATUS_NONFINITE / ZERO_WEIGHT / WEIGHT_SUM (drift above
+ * 1e-4 n) / COLUMN_SUM (relative drift above 1e-5) into the device status word.  Returns, after filling h_stats:
+ * SGP_ERR_ZERO_WEIGHT if a weight is <= 0 or NaN, else SGP_ERR_DEVICE if a kernel of this handle ever gave up a
+ * bounded wait, else SGP_ERR_INVARIANT if any of the three invariants failed, else SGP_OK.  Synchronises.
+ */
+int sgp_check(sgp_handle *h, const float *d_X, const float *d_W, const double *d_colsum_ref, double *h_stats,
+              void *stream);
+
+/*
+ * sgp_get_diagnostics: the diagnostics accumulated by the most recent step taken with option "diagnostics" = 1,
+ * computed inside the fused pass from the tile already on chip (no extra HBM traffic for tau <= 1; tau - 1 extra
+ * ring reads per element otherwise):
+ *   h_param_dev[i] = || h_i - (1/n) sum_j h_j ||_2,  h = x^(k+1/2): the parameter deviation of Sec. 6.1 / Fig. 2,
+ *                    taken after the gradient step and before the mix;
+ *   h_consensus[i] = || z_i^(k+1) - xbar^(k+1) ||_2 with xbar = (1/n) (sum_j x_j + everything in transit): the
+ *                    distance bounded by the consensus lemma of the supplement (definition of xbar after Eq. 4).
+ * Either HOST array (n doubles) may be NULL.  h_summary (HOST, 6 doubles, may be NULL) receives mean, min, max
+ * over nodes of the parameter deviation, then of the consensus distance (the figure plots mean and min..max).
+ * Squares are accumulated in fp32 per warp group, fp64 per CTA and across CTAs.  SGP_ERR_STATE if no such step
+ * was taken.  Synchronises.
+ */
+int sgp_get_diagnostics(sgp_handle *h, double *h_param_dev, double *h_consensus, double *h_summary, void *stream);
 
 /*
  * sgp_param_deviation: the parameter-deviation diagnostic of Sec. 6.1 / Fig. 2.  For an n x ld device
@@ -217,6 +273,15 @@ int sgp_param_deviation(sgp_handle *h, const float *d_A, double *h_dev, void *st
  *                  the bounded wait and the status word can be exercised (that step's results are invalid)
  *   "l2_hint"      L2 evict-first policy on the pipeline's bulk copies: 0 = automatic (gradients only),
  *                  1 = every array, 2 = none, 3 = gradients only, 4 = every array but the gradients
+ *   "send_period"  s >= 1 (default 1): nodes transmit only on steps with k mod s == 0 and keep their whole half step
+ *                  (identity mixing matrix) otherwise -- Alg. 2 lines 5-12 taken literally with s = tau; the c-th
+ *                  transmission uses schedule slot c mod period; messages still arrive tau steps after they were sent
+ *   "diagnostics"  0/1: accumulate the parameter deviation and the consensus distance inside every step
+ *                  (sgp_get_diagnostics reads the latest)
+ *   "check_steps"  0/1, debug: every step is bracketed by an expected-column-sum pre-pass and a column-sum check
+ *                  (sum_i x_i' plus ring against sum_i h_i plus ring, Sec. 2); a drift sets SGP_STATUS_COLUMN_SUM in
+ *                  the device status word.  Costs about two extra passes over the arrays and 8 d bytes of device
+ *                  memory, allocated when the option is switched on (SGP_ERR_ALLOC if that fails)
  * Read-only through sgp_get_option: "last_variant", "last_grid", "last_smem", "last_tile_cols" describe
  * the most recent step launch of the handle (which kernel ran, CTAs, dynamic shared memory, tile width);
  * "launches" counts the step kernels the handle has launched so far.
@@ -239,13 +304,17 @@ int sgp_get_option(const sgp_handle *h, const char *key, int64_t *value);
  * The mixing matrix of the step is passed as HOST arrays in the CSR form sgp_schedule_get produces
  * (h_rowptr[n+1], h_col[nnz], h_val[nnz]; the host-only schedule compiler needs no GPU).  Limits:
  * n <= SGP_MAX_NODES and nnz <= SGP_STATIC_MAX_NNZ, otherwise SGP_ERR_ARG ("use a handle"); a table
- * whose row pointers or column indices are inconsistent returns SGP_ERR_GRAPH.  X, W, M are updated
+ * whose row pointers or column indices are inconsistent, whose senders are not ascending inside a row, that
+ * lacks a self-loop, or whose columns do not sum to one (the schedule compiler's rule) returns SGP_ERR_GRAPH.
+ * X, W, M are updated
  * in place, G is read, Z (may be NULL) is written, exactly as by sgp_step; M may be NULL when
  * momentum == 0.  Asynchronous on `stream`.
  *
  * Set-up: the first call made with a given device current resolves the device address of the static
  * array (cudaGetSymbolAddress) and caches it for that device; make that first call outside any stream
- * capture.  Sharing: all calls on a device use the same array, and it keeps the last call's
+ * capture.  A call whose `stream` is being captured is refused with SGP_ERR_STATE: the table upload reads the
+ * caller's host arrays when it executes, and those are only promised to live for the duration of the call.
+ * Sharing: all calls on a device use the same array, and it keeps the last call's
  * contents; every call rewrites the table and clears the launch words in stream order, so calls
  * issued to ONE stream are safe back to back, while calls that may overlap on the GPU (different
  * streams without a dependency) race and must not be made.
@@ -255,9 +324,10 @@ int sgp_step_static(int n, int64_t d, int64_t ld, const int32_t *h_rowptr, const
                     const float *h_val, int64_t nnz, float *d_X, float *d_W, float *d_M, const float *d_G,
                     float *d_Z, float lr, float momentum, float weight_decay, int nesterov, void *stream);
 
-/* Reads the handle's device status word (0 = no kernel ever gave up a bounded wait; bit 0: consumers gave up
- * waiting for a tile, bit 1: the producer gave up waiting for a free stage, bit 2: copies were still
- * pending at exit).  sgp_reset clears it.  Synchronises. */
+/* Reads the handle's device status word (SGP_STATUS_* bits; 0 = nothing ever went wrong).  Once a wait bit or
+ * the zero-weight bit has been seen by a synchronising call (this one, sgp_check, sgp_step_host), later
+ * sgp_step / sgp_step_adam calls return SGP_ERR_DEVICE / SGP_ERR_ZERO_WEIGHT until sgp_reset, which clears the
+ * word.  Synchronises. */
 int sgp_device_status(sgp_handle *h, unsigned *status);
 /* cudaError_t value latched by the last call that returned SGP_ERR_CUDA on this handle (0 if none). */
 int sgp_last_cuda_error(const sgp_handle *h);

@@ -12,12 +12,17 @@ import os
 import numpy as np
 
 _PKG_DIR = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG_DIR, "libsgp.so")
+# SGP_CHECKED=1 in the environment selects the bounds-checked build of the same library (build.build_checked()).
+LIB_PATH = os.path.join(_PKG_DIR, "libsgp_checked.so" if os.environ.get("SGP_CHECKED", "0") not in ("", "0") else "libsgp.so")
 
 SGP_OK, SGP_ERR_ARG, SGP_ERR_GRAPH, SGP_ERR_CUDA, SGP_ERR_ALLOC, SGP_ERR_STATE, SGP_ERR_DEVICE = 0, -1, -2, -3, -4, -5, -6
+SGP_ERR_ZERO_WEIGHT, SGP_ERR_INVARIANT = -7, -8
+SGP_STATUS_WAIT_TILE, SGP_STATUS_WAIT_STAGE, SGP_STATUS_WAIT_DRAIN, SGP_STATUS_ZERO_WEIGHT = 1, 2, 4, 8
+SGP_STATUS_NONFINITE, SGP_STATUS_WEIGHT_SUM, SGP_STATUS_COLUMN_SUM, SGP_STATUS_BOUNDS = 16, 32, 64, 128
+SGP_FLAG_NONE, SGP_FLAG_BIASED = 0, 1
 SGP_MAX_NODES = 256
 SGP_STATIC_MAX_NNZ = 4096
-SGP_GRAPH_EXP_PEERS, SGP_GRAPH_COMPLETE, SGP_GRAPH_RANDOM_OUTDEG, SGP_GRAPH_CUSTOM = 0, 1, 2, 3
+SGP_GRAPH_EXP_PEERS, SGP_GRAPH_COMPLETE, SGP_GRAPH_RANDOM_OUTDEG, SGP_GRAPH_CUSTOM, SGP_GRAPH_BIPARTITE_EXP = 0, 1, 2, 3, 4
 
 # every symbol include/sgp.h declares
 EXPORTS = [
@@ -25,7 +30,7 @@ EXPORTS = [
     "sgp_create", "sgp_destroy", "sgp_get_schedule", "sgp_step", "sgp_debias", "sgp_step_host", "sgp_reset",
     "sgp_ring_export", "sgp_ring_import", "sgp_check", "sgp_set_option", "sgp_get_option", "sgp_device_status",
     "sgp_last_cuda_error", "sgp_strerror", "sgp_version", "sgp_step_static",
-    "sgp_step_adam", "sgp_param_deviation", "sgp_set_graph",
+    "sgp_step_adam", "sgp_param_deviation", "sgp_set_graph", "sgp_colsum", "sgp_get_diagnostics",
 ]
 
 
@@ -65,11 +70,13 @@ def _load() -> C.CDLL:
         "sgp_step": [vp, vp, vp, vp, vp, vp, i64, f32, f32, f32, i32, vp],
         "sgp_debias": [vp, vp, vp, vp, vp],
         "sgp_step_adam": [vp, vp, vp, vp, vp, vp, vp, i64, i64, f32, f32, f32, f32, f32, vp],
-        "sgp_step_host": [vp, vp, vp, vp, vp, vp, vp, vp, i64, f32, f32, f32, i32, i64],
+        "sgp_step_host": [vp, vp, vp, vp, vp, vp, vp, vp, i64, f32, f32, f32, i32, i64, vp],
         "sgp_reset": [vp, vp],
         "sgp_ring_export": [vp, vp, vp, vp],
         "sgp_ring_import": [vp, vp, vp, vp],
-        "sgp_check": [vp, vp, vp, C.POINTER(C.c_double), vp],
+        "sgp_check": [vp, vp, vp, vp, C.POINTER(C.c_double), vp],
+        "sgp_colsum": [vp, vp, i32, vp, vp],
+        "sgp_get_diagnostics": [vp, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_double), vp],
         "sgp_param_deviation": [vp, vp, C.POINTER(C.c_double), vp],
         "sgp_set_option": [vp, C.c_char_p, i64],
         "sgp_get_option": [vp, C.c_char_p, C.POINTER(i64)],
@@ -130,6 +137,10 @@ class GraphDesc:
     @staticmethod
     def complete() -> "GraphDesc":
         return GraphDesc(SGP_GRAPH_COMPLETE)
+
+    @staticmethod
+    def bipartite_exp() -> "GraphDesc":
+        return GraphDesc(SGP_GRAPH_BIPARTITE_EXP)
 
     @staticmethod
     def random_outdeg(seed: int, num_steps: int, max_outdeg: int = 4) -> "GraphDesc":
@@ -263,10 +274,11 @@ class Sgp:
         _check(_lib.sgp_debias(self._h, _ptr(X), _ptr(W), _ptr(Z), _stream_ptr(stream)), "sgp_debias")
 
     def step_host(self, X, W, M, h_G, h_Z, d_G, d_Z, k: int, lr: float, momentum: float = 0.0,
-                  weight_decay: float = 0.0, nesterov: bool = True, chunk_cols: int = 0) -> None:
+                  weight_decay: float = 0.0, nesterov: bool = True, chunk_cols: int = 0, stream=None) -> None:
         """h_G / h_Z are host (ideally pinned) tensors; everything else lives on the device."""
         _check(_lib.sgp_step_host(self._h, _ptr(X), _ptr(W), _ptr(M), _ptr(h_G), _ptr(h_Z), _ptr(d_G), _ptr(d_Z),
-                                  k, lr, momentum, weight_decay, int(bool(nesterov)), chunk_cols), "sgp_step_host")
+                                  k, lr, momentum, weight_decay, int(bool(nesterov)), chunk_cols,
+                                  _stream_ptr(stream)), "sgp_step_host")
 
     def reset(self, stream=None) -> None:
         _check(_lib.sgp_reset(self._h, _stream_ptr(stream)), "sgp_reset")
@@ -277,11 +289,42 @@ class Sgp:
     def ring_import(self, ring_x, ring_w, stream=None) -> None:
         _check(_lib.sgp_ring_import(self._h, _ptr(ring_x), _ptr(ring_w), _stream_ptr(stream)), "sgp_ring_import")
 
-    def check(self, X, W, stream=None):
-        """(sum of weights incl. in transit, min weight, non-finite count in X, sum of X incl. in transit)."""
-        out = (C.c_double * 4)()
-        _check(_lib.sgp_check(self._h, _ptr(X), _ptr(W), out, _stream_ptr(stream)), "sgp_check")
-        return tuple(out)
+    STAT_NAMES = ("sum_w", "min_w", "nonfinite", "total", "max_colsum_drift", "max_colsum_rel_drift", "sum_w_drift",
+                  "status")
+
+    def check(self, X, W, colsum_ref=None, stream=None, raise_on_error: bool = True):
+        """sgp_check: dict of the eight statistics plus "code" (the call's return code).
+
+        colsum_ref: float64 CUDA tensor of d expected column sums of X plus ring, or None."""
+        import torch
+        if colsum_ref is not None and (colsum_ref.dtype != torch.float64 or not colsum_ref.is_cuda or
+                                       colsum_ref.numel() != self.d or not colsum_ref.is_contiguous()):
+            raise ValueError("colsum_ref must be a contiguous float64 CUDA tensor of d entries")
+        out = (C.c_double * 8)()
+        code = _lib.sgp_check(self._h, _ptr(X), _ptr(W), _ptr(colsum_ref), out, _stream_ptr(stream))
+        if raise_on_error:
+            _check(code, "sgp_check")
+        res = dict(zip(self.STAT_NAMES, out))
+        res["code"] = code
+        return res
+
+    def colsum(self, A, include_ring: bool = False, out=None, stream=None):
+        """sgp_colsum: float64 CUDA tensor of the d column sums of A (plus the ring's when include_ring)."""
+        import torch
+        self._check_mat(A, "A")
+        if out is None:
+            out = torch.empty(self.d, dtype=torch.float64, device=A.device)
+        _check(_lib.sgp_colsum(self._h, _ptr(A), int(bool(include_ring)), _ptr(out), _stream_ptr(stream)), "sgp_colsum")
+        return out
+
+    def diagnostics(self, stream=None):
+        """sgp_get_diagnostics: (param_dev float64[n], consensus float64[n], summary dict of mean/min/max each)."""
+        a = (C.c_double * self.n)()
+        b = (C.c_double * self.n)()
+        s = (C.c_double * 6)()
+        _check(_lib.sgp_get_diagnostics(self._h, a, b, s, _stream_ptr(stream)), "sgp_get_diagnostics")
+        names = ("param_dev_mean", "param_dev_min", "param_dev_max", "consensus_mean", "consensus_min", "consensus_max")
+        return np.array(a[:], dtype=np.float64), np.array(b[:], dtype=np.float64), dict(zip(names, s))
 
     def param_deviation(self, A, stream=None):
         """Per-node distance from the node-wise average row, ||A_i - mean_j A_j||_2 (numpy float64[n])."""
@@ -329,6 +372,8 @@ def graph_desc(w) -> GraphDesc:
         return GraphDesc.exp_peers(w.peers)
     if w.graph == "complete":
         return GraphDesc.complete()
+    if w.graph == "bipartite":
+        return GraphDesc.bipartite_exp()
     if w.graph == "random":
         return GraphDesc.random_outdeg(w.seed, w.num_steps, w.max_outdeg)
     raise ValueError(w.graph)

@@ -58,6 +58,30 @@ OutLists exp_out_lists(int n, int64_t k, int peers) {
   return out;
 }
 
+// Undirected bipartite exponential graph (App. A, "Undirected exponential graph"): odd node i pairs with the even
+// node (i + hop) mod n, hop cycling through 2^1 - 1, 2^2 - 1, ..., 2^floor(log2(n-1)) - 1 (n = 2: the single
+// hop 1); the even node answers, so every step is a perfect matching and P is symmetric.
+std::vector<int> bipartite_hops(int n) {
+  std::vector<int> hops;
+  int top = 0;
+  for (unsigned v = static_cast<unsigned>(n - 1); v > 1; v >>= 1) ++top;   // floor(log2(n-1))
+  for (int j = 1; j <= top; ++j) hops.push_back((1 << j) - 1);
+  if (hops.empty()) hops.push_back(1);
+  return hops;
+}
+
+OutLists bipartite_out_lists(int n, int hop) {
+  OutLists out(static_cast<size_t>(n));
+  for (int i = 0; i < n; ++i) out[static_cast<size_t>(i)].push_back(i);
+  for (int i = 1; i < n; i += 2) {
+    const int j = (i + hop) % n;
+    out[static_cast<size_t>(i)].push_back(j);
+    out[static_cast<size_t>(j)].push_back(i);
+  }
+  for (auto &o : out) sort_unique(o);
+  return out;
+}
+
 OutLists complete_out_lists(int n) {
   OutLists out(static_cast<size_t>(n));
   for (auto &o : out) {
@@ -184,6 +208,11 @@ int sgp_schedule_build(sgp_schedule **out, int n, const sgp_graph_desc *g) {
       case SGP_GRAPH_COMPLETE:
         s->steps.push_back(transpose_uniform(n, complete_out_lists(n)));
         break;
+      case SGP_GRAPH_BIPARTITE_EXP: {
+        if (n < 2 || n % 2 != 0) { rc = SGP_ERR_ARG; break; }     // two halves of equal size
+        for (int hop : bipartite_hops(n)) s->steps.push_back(transpose_uniform(n, bipartite_out_lists(n, hop)));
+        break;
+      }
       case SGP_GRAPH_RANDOM_OUTDEG: {
         if (g->max_outdeg < 1 || g->num_steps < 1 || g->num_steps > (1 << 20)) { rc = SGP_ERR_ARG; break; }
         for (int64_t k = 0; k < g->num_steps; ++k)
@@ -225,6 +254,18 @@ int sgp_schedule_build(sgp_schedule **out, int n, const sgp_graph_desc *g) {
   for (SgpStepCsr &c : s->steps) c.uniform_rows = n > 1 && rows_are_uniform(c, n);
   *out = s;
   return SGP_OK;
+}
+
+SgpStepCsr sgp_identity_step(int n) {
+  SgpStepCsr s;
+  s.rowptr.resize(static_cast<size_t>(n) + 1);
+  s.col.resize(static_cast<size_t>(n));
+  s.val.assign(static_cast<size_t>(n), 1.0f);
+  for (int i = 0; i <= n; ++i) s.rowptr[static_cast<size_t>(i)] = i;
+  for (int i = 0; i < n; ++i) s.col[static_cast<size_t>(i)] = i;
+  s.max_indeg = 1;
+  s.uniform_rows = false;
+  return s;
 }
 
 extern "C" {

@@ -23,3 +23,6 @@ struct sgp_schedule {
 
 // Returns SGP_OK or an error code; *out is a new object on success.
 int sgp_schedule_build(sgp_schedule **out, int n, const sgp_graph_desc *g);
+
+// P = I: the mixing matrix of a step on which no node transmits (Alg. 2 lines 10-11).
+SgpStepCsr sgp_identity_step(int n);

@@ -1,34 +1,40 @@
 // C ABI of the fused SGP step (see include/sgp.h): handle management, argument validation, launch
-// configuration and dispatch.  All arithmetic of the method lives in the kernels.
+// plan and dispatch.  All arithmetic of the method lives in the kernels.
 #include <cuda_runtime.h>
 
 #include <algorithm>
 #include <cmath>
 #include <cstring>
-#include <map>
-#include <mutex>
 #include <new>
 #include <utility>
 #include <vector>
 
 #include "aux_kernels.cuh"
+#include "launch.h"
 #include "schedule.h"
 #include "sgp.h"
-#include "step_kernels.cuh"
 
 using sgp::ConstTable;
 using sgp::StepParams;
+
+namespace {
+constexpr int kDevStatsCheck = 0;                          // kStatCount doubles of sgp_check
+constexpr int kDevStatsDeviation = 8;                      // SGP_MAX_NODES doubles of sgp_param_deviation
+constexpr int kDevStatsDiag = 8 + SGP_MAX_NODES;           // 2 * SGP_MAX_NODES doubles of the fused diagnostics
+constexpr int kDevStatsCount = 8 + 3 * SGP_MAX_NODES;
+constexpr unsigned kWaitBits = sgp::kStatusFullTimeout | sgp::kStatusEmptyTimeout | sgp::kStatusDrainTimeout;
+constexpr double kColumnDriftTol = 1e-5;
+}  // namespace
 
 struct sgp_handle {
   int n = 0;
   int64_t d = 0, ld = 0;
   int tau = 0;
   unsigned flags = 0;
-  int device = 0;
-  int sm_count = 0;
-  int smem_optin = 0;
+  sgp::DeviceInfo dev;
   sgp_schedule *sched = nullptr;
-  // device copy of every slot's CSR, concatenated; offsets in elements
+  SgpStepCsr identity;           // P = I, the mixing matrix of a step without transmissions (send_period > 1)
+  // device copy of every slot's CSR (the schedule's slots, then the identity), concatenated; offsets in elements
   int32_t *d_rowptr = nullptr;
   int32_t *d_col = nullptr;
   float *d_val = nullptr;
@@ -38,12 +44,16 @@ struct sgp_handle {
   float *ring_x = nullptr;   // tau * n * ld
   float *ring_w = nullptr;   // tau * n
   unsigned *d_words = nullptr;  // [0] ticket, [1] status
-  double *d_stats = nullptr;    // 4 doubles for sgp_check, then SGP_MAX_NODES doubles for sgp_param_deviation
+  double *d_stats = nullptr;    // kDevStatsCount doubles
+  double *d_expect = nullptr;   // d doubles, allocated when "check_steps" is switched on
   int64_t opt_variant = 0, opt_tile_cols = 0, opt_ctas_per_sm = 0, opt_stages = 0, opt_l2_hint = 0, opt_single_buffer = 0, opt_wait_limit_ms = 0,
-          opt_inject_stall = 0;
-  int64_t last_variant = 0, last_grid = 0, last_smem = 0, last_tile_cols = 0;   // of the most recent step launch
-  int64_t launches = 0;                                                          // step kernels launched so far
+          opt_inject_stall = 0, opt_send_period = 1, opt_diagnostics = 0, opt_check_steps = 0;
+  sgp::LaunchRecord last;       // of the most recent step launch
+  int64_t launches = 0;         // step kernels launched so far
+  bool diag_valid = false;      // a step with diagnostics has been enqueued since the last reset
+  unsigned seen_status = 0;     // status bits a synchronising call has read back
   cudaStream_t s_h2d = nullptr, s_compute = nullptr, s_d2h = nullptr;
+  cudaEvent_t ev_entry = nullptr;
   std::vector<cudaEvent_t> ev_in, ev_done;
   int last_cuda_error = 0;
   // tensor maps already encoded for (base pointer, box columns)
@@ -71,12 +81,6 @@ namespace {
 
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-inline int floor_log2(int64_t v) {
-  int l = 0;
-  while ((int64_t{1} << (l + 1)) <= v) ++l;
-  return l;
-}
-
 void free_handle(sgp_handle *h) {
   if (h == nullptr) return;
   cudaFree(h->d_rowptr);
@@ -86,76 +90,15 @@ void free_handle(sgp_handle *h) {
   cudaFree(h->ring_w);
   cudaFree(h->d_words);
   cudaFree(h->d_stats);
+  cudaFree(h->d_expect);
   for (cudaEvent_t e : h->ev_in) cudaEventDestroy(e);
   for (cudaEvent_t e : h->ev_done) cudaEventDestroy(e);
+  if (h->ev_entry) cudaEventDestroy(h->ev_entry);
   if (h->s_h2d) cudaStreamDestroy(h->s_h2d);
   if (h->s_compute) cudaStreamDestroy(h->s_compute);
   if (h->s_d2h) cudaStreamDestroy(h->s_d2h);
   delete h->sched;
   delete h;
-}
-
-using StepKernel = void (*)(const StepParams, const ConstTable);
-
-// Per-kernel facts that do not change during the process: registers, static shared memory, and the
-// largest dynamic shared-memory size already enabled (so the attribute calls leave the launch path).
-struct KernelInfo {
-  int num_regs = 0;
-  size_t static_smem = 0;
-  size_t enabled_smem = 48 * 1024;
-};
-std::mutex g_kernel_info_mutex;
-std::map<std::pair<int, const void *>, KernelInfo> g_kernel_info;   // function attributes are per device
-
-int kernel_info(sgp_handle *h, const void *kern, size_t smem, KernelInfo *out) {
-  std::lock_guard<std::mutex> lock(g_kernel_info_mutex);
-  const std::pair<int, const void *> key(h->device, kern);
-  auto it = g_kernel_info.find(key);
-  if (it == g_kernel_info.end()) {
-    cudaFuncAttributes fa;
-    SGP_CUDA_TRY(h, cudaFuncGetAttributes(&fa, kern));
-    KernelInfo ki;
-    ki.num_regs = fa.numRegs;
-    ki.static_smem = fa.sharedSizeBytes;
-    it = g_kernel_info.emplace(key, ki).first;
-  }
-  if (smem > it->second.enabled_smem) {
-    SGP_CUDA_TRY(h, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-    it->second.enabled_smem = smem;
-  }
-  *out = it->second;
-  return SGP_OK;
-}
-
-template <int VEC, int UPD>
-StepKernel pick_regs_flags(bool has_z, bool has_ring) {
-  if (has_z) return has_ring ? sgp::sgp_step_regs_kernel<VEC, UPD, true, true> : sgp::sgp_step_regs_kernel<VEC, UPD, true, false>;
-  return has_ring ? sgp::sgp_step_regs_kernel<VEC, UPD, false, true> : sgp::sgp_step_regs_kernel<VEC, UPD, false, false>;
-}
-template <int VEC>
-StepKernel pick_regs(int upd, bool has_z, bool has_ring) {
-  switch (upd) {
-    case sgp::kUpdSgd: return pick_regs_flags<VEC, sgp::kUpdSgd>(has_z, has_ring);
-    case sgp::kUpdHeavyBall: return pick_regs_flags<VEC, sgp::kUpdHeavyBall>(has_z, has_ring);
-    case sgp::kUpdNesterov: return pick_regs_flags<VEC, sgp::kUpdNesterov>(has_z, has_ring);
-    default: return pick_regs_flags<VEC, sgp::kUpdAdam>(has_z, has_ring);
-  }
-}
-
-using TmaKernel = void (*)(const StepParams, const ConstTable, const sgp::TmaMaps, const int, const int);
-
-template <int UPD>
-TmaKernel pick_tma_flags(bool has_z, bool has_ring) {
-  if (has_z) return has_ring ? sgp::sgp_step_tma_kernel<UPD, true, true> : sgp::sgp_step_tma_kernel<UPD, true, false>;
-  return has_ring ? sgp::sgp_step_tma_kernel<UPD, false, true> : sgp::sgp_step_tma_kernel<UPD, false, false>;
-}
-TmaKernel pick_tma(int upd, bool has_z, bool has_ring) {
-  switch (upd) {
-    case sgp::kUpdSgd: return pick_tma_flags<sgp::kUpdSgd>(has_z, has_ring);
-    case sgp::kUpdHeavyBall: return pick_tma_flags<sgp::kUpdHeavyBall>(has_z, has_ring);
-    case sgp::kUpdNesterov: return pick_tma_flags<sgp::kUpdNesterov>(has_z, has_ring);
-    default: return pick_tma_flags<sgp::kUpdAdam>(has_z, has_ring);
-  }
 }
 
 struct StepArgs {
@@ -174,10 +117,21 @@ inline int update_kind(float momentum, int nesterov) {
   return nesterov != 0 ? sgp::kUpdNesterov : sgp::kUpdHeavyBall;
 }
 
+// Table slot of step k: the c-th transmission (c = k / send_period) uses slot c mod period; a step on which
+// nobody transmits mixes with the identity, stored after the schedule's slots (Alg. 2 lines 5-12).
+inline size_t slot_of(const sgp_handle *h, int64_t k) {
+  const int64_t s = h->opt_send_period;
+  if (k % s != 0) return static_cast<size_t>(h->sched->period());
+  return static_cast<size_t>((k / s) % h->sched->period());
+}
+inline const SgpStepCsr &csr_of(const sgp_handle *h, size_t slot) {
+  return slot == static_cast<size_t>(h->sched->period()) ? h->identity : h->sched->steps[slot];
+}
+
 // Fills the launch-independent part of the kernel arguments for step a.k.
 void fill_params(const sgp_handle *h, const StepArgs &a, int64_t c0, int64_t c1, bool update_w, StepParams *out) {
-  const int64_t slot = a.k % h->sched->period();
-  const SgpStepCsr &csr = h->sched->slot(a.k);
+  const size_t slot = slot_of(h, a.k);
+  const SgpStepCsr &csr = csr_of(h, slot);
   StepParams p{};
   p.X = a.X;
   p.W = a.W;
@@ -194,7 +148,9 @@ void fill_params(const sgp_handle *h, const StepArgs &a, int64_t c0, int64_t c1,
     const int64_t rs = a.k % h->tau;
     p.ring_x = h->ring_x + rs * h->n * h->ld;
     p.ring_w = h->ring_w + rs * h->n;
+    p.ring_base = h->ring_x;
   }
+  p.tau = h->tau;
   p.ld = h->ld;
   p.col_begin = c0;
   p.col_end = c1;
@@ -202,14 +158,16 @@ void fill_params(const sgp_handle *h, const StepArgs &a, int64_t c0, int64_t c1,
   p.nnz = static_cast<int>(csr.col.size());
   p.update_w = update_w ? 1 : 0;
   p.uniform_parts = 0;
+  p.biased = (h->flags & SGP_FLAG_BIASED) ? 1 : 0;
   p.lr = a.lr;
   p.momentum = a.momentum;
   p.wd = a.wd;
-  p.rowptr = h->d_rowptr + h->off_rowptr[static_cast<size_t>(slot)];
-  p.col = h->d_col + h->off_nnz[static_cast<size_t>(slot)];
-  p.val = h->d_val + h->off_nnz[static_cast<size_t>(slot)];
+  p.rowptr = h->d_rowptr + h->off_rowptr[slot];
+  p.col = h->d_col + h->off_nnz[slot];
+  p.val = h->d_val + h->off_nnz[slot];
   p.ticket = h->d_words;
   p.status = h->d_words + 1;
+  p.diag = h->opt_diagnostics ? h->d_stats + kDevStatsDiag : nullptr;
   *out = p;
 }
 
@@ -221,25 +179,6 @@ struct Plan {
   int cps;
 };
 
-// Register-staged kernel: one exchange tile (two barriers per tile) where that keeps the row segments long
-// (n = 64: 1 KB segments 0.95 against 0.92; n = 80: 0.97 against 0.82; n = 96: 512 B 0.92 against 0.89;
-// n > 128: 256 B 0.91 against 0.70); two tiles and one barrier elsewhere (n = 112, 128: 0.94 against 0.92).
-bool auto_single_buffer(int n) { return (n > 32 && n <= 104) || n > 128; }
-
-size_t table_smem_bytes(const sgp_handle *h, int nnz) { return (static_cast<size_t>(h->n) + 1 + 2 * static_cast<size_t>(nnz)) * 4; }
-
-// Tile width of the register-staged kernel (128-bit path): row segments of at least 1 KB and about 2048
-// vector items per tile, shrunk until the exchange tile(s) plus `fixed` bytes stay near 80 KB per CTA --
-// two resident CTAs then leave about half of the SM's 256 KB to the L1 that tracks the loads in flight
-// (measured: n = 48 at 2 x 100 KB reaches 0.74 of the copy bandwidth, at 2 x 50 KB 0.93).
-int64_t regs_tile_cols(const sgp_handle *h, size_t fixed) {
-  int64_t cols = std::max<int64_t>(256, int64_t{4} << floor_log2(std::max<int64_t>(1, 2048 / h->n)));
-  const size_t copies = auto_single_buffer(h->n) ? 1 : 2;
-  const size_t cap = (copies == 1 ? 88 : 80) * 1024;     // n = 80 at 85 KB: 0.97; n = 96 at 102 KB: 0.79
-  while (cols > 32 && copies * static_cast<size_t>(h->n) * cols * 4 + fixed > cap) cols >>= 1;
-  return cols;
-}
-
 // Heuristics from measurements on B200.  The step is HBM-bound; what decides the achieved bandwidth
 // is the length of the contiguous row segments (>= 1 KB), the bytes in flight per SM and a grid that
 // is exactly one wave.  Measured (fraction of the copy bandwidth, rows on 1 KB boundaries):
@@ -250,8 +189,8 @@ int64_t regs_tile_cols(const sgp_handle *h, size_t fixed) {
 Plan make_plan(const sgp_handle *h, int arrays, bool has_m, int nnz, bool vec) {
   Plan pl{1, 0, 2, 0};
   if (vec) {
-    const size_t fixed = 16 * sizeof(uint64_t) + 3 * static_cast<size_t>(h->n) * 4 + 1024 +
-                         (table_smem_bytes(h, nnz) <= 40 * 1024 ? table_smem_bytes(h, nnz) : 0);
+    const size_t table = sgp::table_smem_bytes(h->n, nnz);
+    const size_t fixed = 16 * sizeof(uint64_t) + 3 * static_cast<size_t>(h->n) * 4 + 1024 + (table <= 40 * 1024 ? table : 0);
     const size_t per_kb = static_cast<size_t>(arrays) * h->n * 1024;   // one stage at 1 KB per row segment
     const size_t full_sm = 224 * 1024;
     // The pipelined kernel has ONE consumer group, so its gather is on the critical path: it is only used
@@ -259,7 +198,7 @@ Plan make_plan(const sgp_handle *h, int arrays, bool has_m, int nnz, bool vec) {
     // nine to 0.88, while the register-staged kernel holds 0.98 and 0.95).
     const bool sparse = static_cast<int64_t>(nnz) <= 3 * static_cast<int64_t>(h->n);
     if (!sparse) {
-      pl.tile_cols = regs_tile_cols(h, fixed);
+      pl.tile_cols = sgp::regs_tile_cols(h->n, fixed);
     } else if (!has_m && per_kb >= 24 * 1024 && per_kb <= 40 * 1024) {
       // plain SGD with about 32 KB per stage (n = 16): two CTAs per SM, two stages: 0.98 against 0.97 for the
       // register-staged kernel, which wins at every other n (n = 4: 0.97 against 0.93, n = 32: 0.98 against 0.88)
@@ -270,13 +209,13 @@ Plan make_plan(const sgp_handle *h, int arrays, bool has_m, int nnz, bool vec) {
       // register-staged kernel wins (0.96-0.99 against 0.91-0.95)
       pl = Plan{3, 256, 2, 1};
     } else {
-      pl.tile_cols = regs_tile_cols(h, fixed);
+      pl.tile_cols = sgp::regs_tile_cols(h->n, fixed);
     }
   }
   if (h->opt_variant > 0 && (h->opt_variant == 1) != (pl.variant == 1)) {
     // the caller forces the other kernel family: take that family's defaults
     if (h->opt_variant == 1) {
-      pl = Plan{1, vec ? regs_tile_cols(h, 4 * 1024) : 0, 2, 0};
+      pl = Plan{1, vec ? sgp::regs_tile_cols(h->n, 4 * 1024) : 0, 2, 0};
     } else {
       pl = Plan{static_cast<int>(h->opt_variant), 256, 2, 2};
     }
@@ -288,68 +227,31 @@ Plan make_plan(const sgp_handle *h, int arrays, bool has_m, int nnz, bool vec) {
   return pl;
 }
 
+void record_launch(sgp_handle *h, const sgp::LaunchRecord &rec, int rc) {
+  if (rc == SGP_OK) {
+    h->last = rec;
+    ++h->launches;
+  } else if (rc == SGP_ERR_CUDA) {
+    h->last_cuda_error = rec.cuda_error;
+  }
+}
+
 // One launch of the register-staged kernel over columns [c0, c1) with vector width vec.
 int launch_regs(sgp_handle *h, const StepArgs &a, const Plan &pl, int64_t c0, int64_t c1, int vec, bool update_w,
                 cudaStream_t stream) {
-  const int64_t slot = a.k % h->sched->period();
+  const size_t slot = slot_of(h, a.k);
   StepParams p{};
   fill_params(h, a, c0, c1, update_w, &p);
-
-  // tile width: the plan's, else about four items per thread; at least 128 bytes per row segment
-  const int64_t ncols = c1 - c0;
-  const int min_tv = vec == 4 ? 8 : 32;
-  int64_t tv = int64_t{1} << floor_log2(std::max<int64_t>(1, sgp::kThreads * 4 / h->n));
-  if (pl.tile_cols > 0) tv = int64_t{1} << floor_log2(std::max<int64_t>(1, pl.tile_cols / vec));
-  tv = std::max<int64_t>(tv, min_tv);
-  // short rows: narrower tiles until there is about a tile per SM (launch-latency regime)
-  if (h->opt_tile_cols == 0)
-    while (tv > min_tv && tv * vec > 128 && (ncols + tv * vec - 1) / (tv * vec) < h->sm_count) tv >>= 1;
-  const size_t table_bytes = table_smem_bytes(h, p.nnz);
-  if (h->const_ok[static_cast<size_t>(slot)]) p.table_mode = 0;
-  else p.table_mode = table_bytes <= 40 * 1024 ? 1 : 2;
-  const bool uniform = h->tau == 0 && h->sched->slot(a.k).uniform_rows;
-  // large n: one exchange tile (two barriers per tile) so that the row segments can stay twice as long
-  p.single_buffer = h->opt_single_buffer == 1 ? 1 : (h->opt_single_buffer == 2 ? 0 : (auto_single_buffer(h->n) ? 1 : 0));
-  size_t smem = 0;
-  for (;;) {
-    p.uniform_parts = uniform ? static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(8, sgp::kThreads / tv))) : 0;
-    smem = (p.single_buffer ? 1 : 2) * static_cast<size_t>(h->n) * tv * vec * 4 + 3 * static_cast<size_t>(h->n) * 4 +
-           static_cast<size_t>(p.uniform_parts) * tv * vec * 4 + (p.table_mode < 2 ? table_bytes : 0);
-    if (smem <= 110 * 1024 || tv <= min_tv) break;
-    tv >>= 1;
-  }
-  if (smem > static_cast<size_t>(h->smem_optin)) return SGP_ERR_ARG;
-  p.log2_tile_vecs = floor_log2(tv);
-  const int64_t tile_cols = tv * vec;
-  const int64_t ntiles = (ncols + tile_cols - 1) / tile_cols;
-  StepKernel kern = vec == 4 ? pick_regs<4>(a.upd, a.Z != nullptr, h->tau > 0)
-                             : pick_regs<1>(a.upd, a.Z != nullptr, h->tau > 0);
-  KernelInfo ki;
-  {
-    const int rc = kernel_info(h, reinterpret_cast<const void *>(kern), smem, &ki);
-    if (rc != SGP_OK) return rc;
-  }
-  int cps = pl.cps;
-  if (cps <= 0) {
-    // Persistent grid of exactly one wave: CTAs resident per SM by registers, shared memory and threads.
-    // (Computed here rather than asked of the occupancy calculator, whose answer depends on the
-    // shared-memory carve-out it assumes; the hardware picks the carve-out that fits the launch.)
-    const int regs_per_cta = ((ki.num_regs + 7) / 8 * 8) * sgp::kThreads;
-    const int by_regs = regs_per_cta > 0 ? 65536 / regs_per_cta : 8;
-    const int by_smem = static_cast<int>((227 * 1024) / (smem + ki.static_smem + 1024));
-    cps = std::max(1, std::min({by_regs, by_smem, 2048 / sgp::kThreads}));
-  }
-  const int64_t grid = std::min<int64_t>(ntiles, static_cast<int64_t>(h->sm_count) * cps);
-  static const ConstTable kEmptyTable{};
-  const ConstTable &ct = p.table_mode == 0 ? h->const_tables[static_cast<size_t>(slot)] : kEmptyTable;
-  kern<<<static_cast<unsigned>(grid), sgp::kThreads, smem, stream>>>(p, ct);
-  SGP_CUDA_TRY(h, cudaGetLastError());
-  h->last_variant = 1;
-  ++h->launches;
-  h->last_grid = grid;
-  h->last_smem = static_cast<int64_t>(smem);
-  h->last_tile_cols = tile_cols;
-  return SGP_OK;
+  sgp::RegsOptions opt;
+  opt.tile_cols = pl.tile_cols;
+  opt.tile_cols_forced = h->opt_tile_cols > 0;
+  opt.cps = pl.cps;
+  opt.single_buffer = static_cast<int>(h->opt_single_buffer);
+  sgp::LaunchRecord rec;
+  const int rc = sgp::launch_regs(h->dev, p, h->const_ok[slot] ? &h->const_tables[slot] : nullptr, a.upd, vec,
+                                  csr_of(h, slot).uniform_rows, opt, stream, &rec);
+  record_launch(h, rec, rc);
+  return rc;
 }
 
 using EncodeTiledFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
@@ -358,7 +260,8 @@ using EncodeTiledFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_
 
 // Tensor map of an n x d fp32 array with row pitch ld whose box is (box_cols x n); cached per pointer.
 // Returns false when the driver entry point is unavailable or the encoding is rejected.
-bool get_tensor_map(sgp_handle *h, const float *base, int box_cols, CUtensorMap *out) {
+bool get_tensor_map(void *ctx, const float *base, int box_cols, CUtensorMap *out) {
+  sgp_handle *h = static_cast<sgp_handle *>(ctx);
   for (const auto &e : h->map_cache)
     if (e.ptr == base && e.box_cols == box_cols) {
       *out = e.map;
@@ -396,62 +299,24 @@ bool get_tensor_map(sgp_handle *h, const float *base, int box_cols, CUtensorMap 
 // the register-staged kernel.
 int launch_tma(sgp_handle *h, const StepArgs &a, const Plan &pl, int64_t c0, int64_t c1, bool update_w,
                cudaStream_t stream) {
-  const int64_t slot = a.k % h->sched->period();
+  const size_t slot = slot_of(h, a.k);
   StepParams p{};
   fill_params(h, a, c0, c1, update_w, &p);
-  const bool has_m = a.M != nullptr, has_v = a.V != nullptr, has_ring = h->tau > 0;
-  const int arrays = 2 + (has_m ? 1 : 0) + (has_v ? 1 : 0) + (has_ring ? 1 : 0);
-  int64_t tv = int64_t{1} << floor_log2(std::max<int64_t>(1, (pl.tile_cols > 0 ? pl.tile_cols : 256) / 4));
-  tv = std::max<int64_t>(tv, 8);
-  int stages = std::max(1, pl.stages);
-  const int cps = pl.cps > 0 ? pl.cps : 2;
-  const size_t table_bytes = table_smem_bytes(h, p.nnz);
-  if (h->const_ok[static_cast<size_t>(slot)]) p.table_mode = 0;
-  else p.table_mode = table_bytes <= 40 * 1024 ? 1 : 2;
-  const bool uniform = h->tau == 0 && h->sched->slot(a.k).uniform_rows;
-  size_t fixed = 16 * sizeof(uint64_t) + 3 * static_cast<size_t>(h->n) * 4 + (p.table_mode < 2 ? table_bytes : 0);
-  const size_t budget = std::min<size_t>(static_cast<size_t>(h->smem_optin), (228 * 1024) / static_cast<size_t>(cps) - 2048);
-  size_t smem = 0;
-  for (;;) {
-    p.uniform_parts = uniform ? static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(8, sgp::kTmaConsumers / tv))) : 0;
-    smem = static_cast<size_t>(stages) * arrays * h->n * tv * 16 + fixed + static_cast<size_t>(p.uniform_parts) * tv * 16;
-    if (smem <= budget) break;
-    if (h->opt_stages == 0 && stages > 2) --stages;
-    else if (h->opt_tile_cols == 0 && tv > 8) tv >>= 1;
-    else return SGP_ERR_STATE;
-  }
-  p.log2_tile_vecs = floor_log2(tv);
-  const int64_t tile_cols = tv * 4;
-  const int64_t ntiles = (c1 - c0 + tile_cols - 1) / tile_cols;
-  const int64_t grid = std::min<int64_t>(ntiles, static_cast<int64_t>(h->sm_count) * cps);
-  p.wait_limit_ms = h->opt_wait_limit_ms > 0 ? static_cast<int>(h->opt_wait_limit_ms) : 2000;
-  p.inject_stall = h->opt_inject_stall ? 1 : 0;
-  p.l2_hint = h->opt_l2_hint == 2 ? 0 : (h->opt_l2_hint == 0 ? 3 : static_cast<int>(h->opt_l2_hint));
-  TmaKernel kern = pick_tma(a.upd, a.Z != nullptr, has_ring);
-  {
-    KernelInfo ki;
-    const int rc = kernel_info(h, reinterpret_cast<const void *>(kern), smem, &ki);
-    if (rc != SGP_OK) return rc;
-  }
-  static const ConstTable kEmptyTable{};
-  const ConstTable &ct = p.table_mode == 0 ? h->const_tables[static_cast<size_t>(slot)] : kEmptyTable;
-  // 2-D tensor maps (one copy per array per tile) when the box fits; else one bulk copy per row segment
-  sgp::TmaMaps maps;
-  std::memset(&maps, 0, sizeof(maps));
-  bool use_maps = pl.variant == 2 && tile_cols <= 256 && tile_cols * 4 % 128 == 0;
-  if (use_maps) use_maps = get_tensor_map(h, a.X, static_cast<int>(tile_cols), &maps.x);
-  if (use_maps) use_maps = get_tensor_map(h, a.G, static_cast<int>(tile_cols), &maps.g);
-  if (use_maps && has_m) use_maps = get_tensor_map(h, a.M, static_cast<int>(tile_cols), &maps.m);
-  if (use_maps && has_v) use_maps = get_tensor_map(h, a.V, static_cast<int>(tile_cols), &maps.v);
-  if (use_maps && has_ring) use_maps = get_tensor_map(h, p.ring_x, static_cast<int>(tile_cols), &maps.r);
-  kern<<<static_cast<unsigned>(grid), sgp::kTmaThreads, smem, stream>>>(p, ct, maps, stages, use_maps ? 1 : 0);
-  SGP_CUDA_TRY(h, cudaGetLastError());
-  h->last_variant = use_maps ? 2 : 3;
-  ++h->launches;
-  h->last_grid = grid;
-  h->last_smem = static_cast<int64_t>(smem);
-  h->last_tile_cols = tile_cols;
-  return SGP_OK;
+  sgp::TmaOptions opt;
+  opt.variant = pl.variant;
+  opt.tile_cols = pl.tile_cols > 0 ? pl.tile_cols : 256;
+  opt.tile_cols_forced = h->opt_tile_cols > 0;
+  opt.stages = pl.stages;
+  opt.stages_forced = h->opt_stages > 0;
+  opt.cps = pl.cps > 0 ? pl.cps : 2;
+  opt.wait_limit_ms = h->opt_wait_limit_ms > 0 ? static_cast<int>(h->opt_wait_limit_ms) : 2000;
+  opt.inject_stall = h->opt_inject_stall ? 1 : 0;
+  opt.l2_hint = h->opt_l2_hint == 2 ? 0 : (h->opt_l2_hint == 0 ? 3 : static_cast<int>(h->opt_l2_hint));
+  sgp::LaunchRecord rec;
+  const int rc = sgp::launch_tma(h->dev, p, h->const_ok[slot] ? &h->const_tables[slot] : nullptr, a.upd,
+                                 csr_of(h, slot).uniform_rows, opt, get_tensor_map, h, stream, &rec);
+  record_launch(h, rec, rc);
+  return rc;
 }
 
 // The whole step over columns [c0, c1): 128-bit kernel on the aligned bulk, scalar kernel on what is left.
@@ -461,11 +326,11 @@ int launch_step_range(sgp_handle *h, const StepArgs &a, int64_t c0, int64_t c1, 
                       (c0 % 4 == 0);
   const int64_t vec_end = vec_ok ? c0 + ((c1 - c0) & ~int64_t{3}) : c0;
   const int arrays = 2 + (a.M != nullptr ? 1 : 0) + (a.V != nullptr ? 1 : 0) + (h->tau > 0 ? 1 : 0);
-  const int nnz = static_cast<int>(h->sched->slot(a.k).col.size());
+  const int nnz = static_cast<int>(csr_of(h, slot_of(h, a.k)).col.size());
   if (vec_end > c0) {
     Plan pl = make_plan(h, arrays, a.M != nullptr, nnz, true);
     // short rows (fewer 1 KB tiles than SMs): the register kernel with narrow tiles spreads them better
-    if (h->opt_variant == 0 && pl.variant >= 2 && (vec_end - c0) < int64_t{256} * h->sm_count) pl = Plan{1, 256, 2, 0};
+    if (h->opt_variant == 0 && pl.variant >= 2 && (vec_end - c0) < int64_t{256} * h->dev.sm_count) pl = Plan{1, 256, 2, 0};
     int rc = SGP_ERR_STATE;
     if (pl.variant >= 2) rc = launch_tma(h, a, pl, c0, vec_end, update_w && vec_end == c1, stream);
     if (rc == SGP_ERR_STATE) {
@@ -479,6 +344,62 @@ int launch_step_range(sgp_handle *h, const StepArgs &a, int64_t c0, int64_t c1, 
   return SGP_OK;
 }
 
+unsigned column_grid(const sgp_handle *h) {
+  return static_cast<unsigned>(std::max<int64_t>(1, std::min<int64_t>((h->d + 255) / 256, static_cast<int64_t>(h->dev.sm_count) * 8)));
+}
+
+// Debug pre-pass of a checked step: what every column of X plus ring must sum to after the step.
+int launch_expected(sgp_handle *h, const StepArgs &a, cudaStream_t st) {
+  const sgp::UpdateScalars us{a.lr, a.momentum, a.wd, a.beta1, a.beta2, a.eps, a.adam_step, a.adam_rsqrt_bc2};
+  const unsigned grid = column_grid(h);
+  const int ring_rows = h->tau * h->n;
+  switch (a.upd) {
+    case sgp::kUpdSgd:
+      sgp::sgp_expected_colsum_kernel<sgp::kUpdSgd><<<grid, 256, 0, st>>>(a.X, a.G, a.M, a.V, h->n, h->d, h->ld, us, h->ring_x, ring_rows, h->d_expect);
+      break;
+    case sgp::kUpdHeavyBall:
+      sgp::sgp_expected_colsum_kernel<sgp::kUpdHeavyBall><<<grid, 256, 0, st>>>(a.X, a.G, a.M, a.V, h->n, h->d, h->ld, us, h->ring_x, ring_rows, h->d_expect);
+      break;
+    case sgp::kUpdNesterov:
+      sgp::sgp_expected_colsum_kernel<sgp::kUpdNesterov><<<grid, 256, 0, st>>>(a.X, a.G, a.M, a.V, h->n, h->d, h->ld, us, h->ring_x, ring_rows, h->d_expect);
+      break;
+    default:
+      sgp::sgp_expected_colsum_kernel<sgp::kUpdAdam><<<grid, 256, 0, st>>>(a.X, a.G, a.M, a.V, h->n, h->d, h->ld, us, h->ring_x, ring_rows, h->d_expect);
+  }
+  SGP_CUDA_TRY(h, cudaGetLastError());
+  return SGP_OK;
+}
+
+// Enqueues the invariant scan of (X, W, ring) against an optional column-sum reference; statistics stay on the
+// device (d_stats) and violations are ORed into the status word.  No synchronisation.
+int enqueue_check(sgp_handle *h, const float *X, const float *W, const double *ref, cudaStream_t st) {
+  double *stats = h->d_stats + kDevStatsCheck;
+  SGP_CUDA_TRY(h, cudaMemsetAsync(stats, 0, sgp::kStatCount * sizeof(double), st));
+  sgp::sgp_colsum_kernel<<<column_grid(h), 256, 0, st>>>(X, h->n, h->d, h->ld, h->ring_x, h->tau * h->n, nullptr, ref, stats);
+  sgp::sgp_weight_scan_kernel<<<1, 256, 0, st>>>(W, h->n, h->ring_w, h->tau * h->n, stats);
+  sgp::sgp_check_finalize_kernel<<<1, 1, 0, st>>>(stats, h->n, 1, ref != nullptr ? 1 : 0, kColumnDriftTol, h->d_words + 1);
+  SGP_CUDA_TRY(h, cudaGetLastError());
+  return SGP_OK;
+}
+
+// A whole step on the device arrays: optional debug bracket, optional diagnostics, the fused launch(es).
+int run_step(sgp_handle *h, const StepArgs &a, cudaStream_t st) {
+  if (h->seen_status & kWaitBits) return SGP_ERR_DEVICE;
+  if (h->seen_status & sgp::kStatusZeroWeight) return SGP_ERR_ZERO_WEIGHT;
+  if (h->opt_check_steps) {
+    const int rc = launch_expected(h, a, st);
+    if (rc != SGP_OK) return rc;
+  }
+  if (h->opt_diagnostics) {
+    SGP_CUDA_TRY(h, cudaMemsetAsync(h->d_stats + kDevStatsDiag, 0, 2 * static_cast<size_t>(h->n) * sizeof(double), st));
+    h->diag_valid = true;
+  }
+  const int rc = launch_step_range(h, a, 0, h->d, true, st);
+  if (rc != SGP_OK) return rc;
+  if (h->opt_check_steps) return enqueue_check(h, a.X, a.W, h->d_expect, st);
+  return SGP_OK;
+}
+
 // The handle's tables and ring live on the device that was current at sgp_create.
 int check_device(const sgp_handle *h) {
   int dev = -1;
@@ -486,7 +407,7 @@ int check_device(const sgp_handle *h) {
     (void)cudaGetLastError();
     return SGP_ERR_CUDA;
   }
-  return dev == h->device ? SGP_OK : SGP_ERR_STATE;
+  return dev == h->dev.device ? SGP_OK : SGP_ERR_STATE;
 }
 
 int validate_step(const sgp_handle *h, const float *X, const float *W, const float *M, const float *G, int64_t k,
@@ -496,16 +417,18 @@ int validate_step(const sgp_handle *h, const float *X, const float *W, const flo
   return check_device(h);
 }
 
-// Builds the device tables of a compiled schedule and installs them (and the schedule) in the handle,
-// releasing whatever the handle held before.  The caller guarantees that no kernel still reads the old tables.
+// Builds the device tables of a compiled schedule (plus the identity step) and installs them (and the schedule)
+// in the handle, releasing whatever the handle held before.  The caller guarantees that no kernel still reads
+// the old tables.
 int upload_schedule(sgp_handle *h, sgp_schedule *sched) {
   std::vector<int32_t> rowptr, col;
   std::vector<float> val;
   std::vector<int64_t> off_rowptr, off_nnz;
   std::vector<ConstTable> const_tables;
   std::vector<char> const_ok;
-  for (int64_t s = 0; s < sched->period(); ++s) {
-    const SgpStepCsr &c = sched->steps[static_cast<size_t>(s)];
+  const SgpStepCsr identity = sgp_identity_step(h->n);
+  for (int64_t s = 0; s <= sched->period(); ++s) {
+    const SgpStepCsr &c = s < sched->period() ? sched->steps[static_cast<size_t>(s)] : identity;
     off_rowptr.push_back(static_cast<int64_t>(rowptr.size()));
     off_nnz.push_back(static_cast<int64_t>(col.size()));
     rowptr.insert(rowptr.end(), c.rowptr.begin(), c.rowptr.end());
@@ -551,8 +474,18 @@ int upload_schedule(sgp_handle *h, sgp_schedule *sched) {
   h->off_nnz.swap(off_nnz);
   h->const_tables.swap(const_tables);
   h->const_ok.swap(const_ok);
+  h->identity = identity;
   if (h->sched != sched) delete h->sched;
   h->sched = sched;
+  return SGP_OK;
+}
+
+// Reads the device status word back (the stream must already be synchronised) and remembers what it saw.
+int refresh_status(sgp_handle *h, unsigned *out) {
+  unsigned v = 0;
+  SGP_CUDA_TRY(h, cudaMemcpy(&v, h->d_words + 1, sizeof(unsigned), cudaMemcpyDeviceToHost));
+  h->seen_status |= v;
+  if (out) *out = v;
   return SGP_OK;
 }
 
@@ -560,7 +493,7 @@ int upload_schedule(sgp_handle *h, sgp_schedule *sched) {
 
 extern "C" {
 
-int sgp_version(void) { return 100; }
+int sgp_version(void) { return 200; }
 
 const char *sgp_strerror(int code) {
   switch (code) {
@@ -571,6 +504,8 @@ const char *sgp_strerror(int code) {
     case SGP_ERR_ALLOC: return "allocation failed";
     case SGP_ERR_STATE: return "call not valid for this handle";
     case SGP_ERR_DEVICE: return "a kernel gave up a bounded wait";
+    case SGP_ERR_ZERO_WEIGHT: return "a push-sum weight is not positive";
+    case SGP_ERR_INVARIANT: return "an invariant of column-stochastic mixing does not hold";
     default: return "unknown error";
   }
 }
@@ -578,7 +513,7 @@ const char *sgp_strerror(int code) {
 int sgp_create(sgp_handle **out, int n, int64_t d, int64_t ld, const sgp_graph_desc *g, int tau, unsigned flags) {
   if (out == nullptr) return SGP_ERR_ARG;
   *out = nullptr;
-  if (n < 1 || n > SGP_MAX_NODES || d < 1 || ld < d || tau < 0 || tau > 64 || g == nullptr || flags != SGP_FLAG_NONE)
+  if (n < 1 || n > SGP_MAX_NODES || d < 1 || ld < d || tau < 0 || tau > 64 || g == nullptr || (flags & ~SGP_FLAG_BIASED) != 0)
     return SGP_ERR_ARG;
   sgp_schedule *sched = nullptr;
   int rc = sgp_schedule_build(&sched, n, g);
@@ -595,42 +530,30 @@ int sgp_create(sgp_handle **out, int n, int64_t d, int64_t ld, const sgp_graph_d
   h->flags = flags;
   h->sched = sched;
 
-  auto fail = [&](int code, cudaError_t e) {
-    const int err = static_cast<int>(e);
+  auto fail = [&](int code) {
     free_handle(h);
     (void)cudaGetLastError();
-    (void)err;
     return code;
   };
-  cudaError_t e = cudaGetDevice(&h->device);
-  if (e != cudaSuccess) return fail(SGP_ERR_CUDA, e);
-  e = cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device);
-  if (e != cudaSuccess) return fail(SGP_ERR_CUDA, e);
-  e = cudaDeviceGetAttribute(&h->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, h->device);
-  if (e != cudaSuccess) return fail(SGP_ERR_CUDA, e);
-
+  if (cudaGetDevice(&h->dev.device) != cudaSuccess) return fail(SGP_ERR_CUDA);
+  if (cudaDeviceGetAttribute(&h->dev.sm_count, cudaDevAttrMultiProcessorCount, h->dev.device) != cudaSuccess) return fail(SGP_ERR_CUDA);
+  if (cudaDeviceGetAttribute(&h->dev.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, h->dev.device) != cudaSuccess)
+    return fail(SGP_ERR_CUDA);
   {
     const int rc_up = upload_schedule(h, sched);
-    if (rc_up != SGP_OK) return fail(rc_up, cudaSuccess);
+    if (rc_up != SGP_OK) return fail(rc_up);
   }
-  e = cudaMalloc(&h->d_words, 2 * sizeof(unsigned));
-  if (e != cudaSuccess) return fail(SGP_ERR_ALLOC, e);
-  e = cudaMalloc(&h->d_stats, (4 + SGP_MAX_NODES) * sizeof(double));
-  if (e != cudaSuccess) return fail(SGP_ERR_ALLOC, e);
+  if (cudaMalloc(&h->d_words, 2 * sizeof(unsigned)) != cudaSuccess) return fail(SGP_ERR_ALLOC);
+  if (cudaMalloc(&h->d_stats, kDevStatsCount * sizeof(double)) != cudaSuccess) return fail(SGP_ERR_ALLOC);
   if (tau > 0) {
-    e = cudaMalloc(&h->ring_x, static_cast<size_t>(tau) * n * ld * sizeof(float));
-    if (e != cudaSuccess) return fail(SGP_ERR_ALLOC, e);
-    e = cudaMalloc(&h->ring_w, static_cast<size_t>(tau) * n * sizeof(float));
-    if (e != cudaSuccess) return fail(SGP_ERR_ALLOC, e);
-    e = cudaMemset(h->ring_x, 0, static_cast<size_t>(tau) * n * ld * sizeof(float));
-    if (e != cudaSuccess) return fail(SGP_ERR_CUDA, e);
-    e = cudaMemset(h->ring_w, 0, static_cast<size_t>(tau) * n * sizeof(float));
-    if (e != cudaSuccess) return fail(SGP_ERR_CUDA, e);
+    if (cudaMalloc(&h->ring_x, static_cast<size_t>(tau) * n * ld * sizeof(float)) != cudaSuccess) return fail(SGP_ERR_ALLOC);
+    if (cudaMalloc(&h->ring_w, static_cast<size_t>(tau) * n * sizeof(float)) != cudaSuccess) return fail(SGP_ERR_ALLOC);
+    if (cudaMemset(h->ring_x, 0, static_cast<size_t>(tau) * n * ld * sizeof(float)) != cudaSuccess) return fail(SGP_ERR_CUDA);
+    if (cudaMemset(h->ring_w, 0, static_cast<size_t>(tau) * n * sizeof(float)) != cudaSuccess) return fail(SGP_ERR_CUDA);
   }
-  e = cudaMemset(h->d_words, 0, 2 * sizeof(unsigned));
-  if (e != cudaSuccess) return fail(SGP_ERR_CUDA, e);
-  e = cudaDeviceSynchronize();
-  if (e != cudaSuccess) return fail(SGP_ERR_CUDA, e);
+  if (cudaMemset(h->d_words, 0, 2 * sizeof(unsigned)) != cudaSuccess) return fail(SGP_ERR_CUDA);
+  if (cudaMemset(h->d_stats, 0, kDevStatsCount * sizeof(double)) != cudaSuccess) return fail(SGP_ERR_CUDA);
+  if (cudaDeviceSynchronize() != cudaSuccess) return fail(SGP_ERR_CUDA);
   *out = h;
   return SGP_OK;
 }
@@ -667,7 +590,7 @@ int sgp_step(sgp_handle *h, float *d_X, float *d_W, float *d_M, const float *d_G
   if (rc != SGP_OK) return rc;
   const StepArgs a{d_X, d_W, momentum != 0.0f ? d_M : nullptr, d_G, d_Z, k, lr, momentum, weight_decay,
                    update_kind(momentum, nesterov)};
-  return launch_step_range(h, a, 0, h->d, true, static_cast<cudaStream_t>(stream));
+  return run_step(h, a, static_cast<cudaStream_t>(stream));
 }
 
 int sgp_step_adam(sgp_handle *h, float *d_X, float *d_W, float *d_M1, float *d_M2, const float *d_G, float *d_Z,
@@ -686,7 +609,7 @@ int sgp_step_adam(sgp_handle *h, float *d_X, float *d_W, float *d_M1, float *d_M
   const double bc2 = 1.0 - std::pow(static_cast<double>(beta2), static_cast<double>(t));
   a.adam_step = static_cast<float>(static_cast<double>(lr) / bc1);
   a.adam_rsqrt_bc2 = static_cast<float>(1.0 / std::sqrt(bc2));
-  return launch_step_range(h, a, 0, h->d, true, static_cast<cudaStream_t>(stream));
+  return run_step(h, a, static_cast<cudaStream_t>(stream));
 }
 
 int sgp_debias(sgp_handle *h, const float *d_X, const float *d_W, float *d_Z, void *stream) {
@@ -694,25 +617,29 @@ int sgp_debias(sgp_handle *h, const float *d_X, const float *d_W, float *d_Z, vo
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool vec_ok = aligned16(d_X) && aligned16(d_Z) && (h->ld % 4 == 0);
   const int64_t work = vec_ok ? (h->d + 3) / 4 : h->d;
-  const int64_t per_row = std::max<int64_t>(1, (static_cast<int64_t>(h->sm_count) * 8 + h->n - 1) / h->n);
+  const int64_t per_row = std::max<int64_t>(1, (static_cast<int64_t>(h->dev.sm_count) * 8 + h->n - 1) / h->n);
   const unsigned gx = static_cast<unsigned>(std::max<int64_t>(1, std::min<int64_t>((work + 255) / 256, per_row)));
   const dim3 grid(gx, static_cast<unsigned>(h->n));
-  if (vec_ok) sgp::sgp_debias_kernel<4><<<grid, 256, 0, st>>>(d_X, d_W, d_Z, h->d, h->ld);
-  else sgp::sgp_debias_kernel<1><<<grid, 256, 0, st>>>(d_X, d_W, d_Z, h->d, h->ld);
+  const int biased = (h->flags & SGP_FLAG_BIASED) ? 1 : 0;
+  if (vec_ok) sgp::sgp_debias_kernel<4><<<grid, 256, 0, st>>>(d_X, d_W, d_Z, h->d, h->ld, biased, h->d_words + 1);
+  else sgp::sgp_debias_kernel<1><<<grid, 256, 0, st>>>(d_X, d_W, d_Z, h->d, h->ld, biased, h->d_words + 1);
   SGP_CUDA_TRY(h, cudaGetLastError());
   return SGP_OK;
 }
 
 int sgp_step_host(sgp_handle *h, float *d_X, float *d_W, float *d_M, const float *h_G, float *h_Z, float *d_G,
                   float *d_Z, int64_t k, float lr, float momentum, float weight_decay, int nesterov,
-                  int64_t chunk_cols) {
+                  int64_t chunk_cols, void *stream) {
   int rc = validate_step(h, d_X, d_W, d_M, d_G, k, momentum);
   if (rc != SGP_OK) return rc;
   if (h_G == nullptr || (h_Z != nullptr && d_Z == nullptr)) return SGP_ERR_ARG;
+  if (h->seen_status & kWaitBits) return SGP_ERR_DEVICE;
+  if (h->seen_status & sgp::kStatusZeroWeight) return SGP_ERR_ZERO_WEIGHT;
   if (h->s_h2d == nullptr) {
     SGP_CUDA_TRY(h, cudaStreamCreateWithFlags(&h->s_h2d, cudaStreamNonBlocking));
     SGP_CUDA_TRY(h, cudaStreamCreateWithFlags(&h->s_compute, cudaStreamNonBlocking));
     SGP_CUDA_TRY(h, cudaStreamCreateWithFlags(&h->s_d2h, cudaStreamNonBlocking));
+    SGP_CUDA_TRY(h, cudaEventCreateWithFlags(&h->ev_entry, cudaEventDisableTiming));
   }
   // default chunk: about 64 MB of gradient per chunk, a multiple of 1024 columns
   if (chunk_cols <= 0) chunk_cols = std::max<int64_t>(1024, (int64_t{64} << 20) / (4 * h->n) / 1024 * 1024);
@@ -725,10 +652,18 @@ int sgp_step_host(sgp_handle *h, float *d_X, float *d_W, float *d_M, const float
     SGP_CUDA_TRY(h, cudaEventCreateWithFlags(&b, cudaEventDisableTiming));
     h->ev_done.push_back(b);
   }
-  // earlier work of the caller on the legacy/default stream must be visible
-  SGP_CUDA_TRY(h, cudaDeviceSynchronize());
+  // what the caller already enqueued on its stream (it may produce X, W, M or read d_G, d_Z) comes first:
+  // an event wait on the device, not a host synchronisation
+  SGP_CUDA_TRY(h, cudaEventRecord(h->ev_entry, static_cast<cudaStream_t>(stream)));
+  SGP_CUDA_TRY(h, cudaStreamWaitEvent(h->s_h2d, h->ev_entry, 0));
+  SGP_CUDA_TRY(h, cudaStreamWaitEvent(h->s_compute, h->ev_entry, 0));
+  SGP_CUDA_TRY(h, cudaStreamWaitEvent(h->s_d2h, h->ev_entry, 0));
   const StepArgs a{d_X, d_W, momentum != 0.0f ? d_M : nullptr, d_G, h_Z != nullptr ? d_Z : nullptr,
                    k, lr, momentum, weight_decay, update_kind(momentum, nesterov)};
+  if (h->opt_diagnostics) {
+    SGP_CUDA_TRY(h, cudaMemsetAsync(h->d_stats + kDevStatsDiag, 0, 2 * static_cast<size_t>(h->n) * sizeof(double), h->s_compute));
+    h->diag_valid = true;
+  }
   const size_t pitch = static_cast<size_t>(h->ld) * sizeof(float);
   for (int64_t c = 0; c < nchunks; ++c) {
     const int64_t c0 = c * chunk_cols, c1 = std::min(h->d, c0 + chunk_cols);
@@ -749,7 +684,7 @@ int sgp_step_host(sgp_handle *h, float *d_X, float *d_W, float *d_M, const float
   SGP_CUDA_TRY(h, cudaStreamSynchronize(h->s_h2d));
   SGP_CUDA_TRY(h, cudaStreamSynchronize(h->s_compute));
   SGP_CUDA_TRY(h, cudaStreamSynchronize(h->s_d2h));
-  return SGP_OK;
+  return refresh_status(h, nullptr);
 }
 
 int sgp_reset(sgp_handle *h, void *stream) {
@@ -760,6 +695,8 @@ int sgp_reset(sgp_handle *h, void *stream) {
     SGP_CUDA_TRY(h, cudaMemsetAsync(h->ring_w, 0, static_cast<size_t>(h->tau) * h->n * sizeof(float), st));
   }
   SGP_CUDA_TRY(h, cudaMemsetAsync(h->d_words, 0, 2 * sizeof(unsigned), st));
+  h->seen_status = 0;
+  h->diag_valid = false;
   return SGP_OK;
 }
 
@@ -785,39 +722,94 @@ int sgp_ring_import(sgp_handle *h, const float *d_ring_x, const float *d_ring_w,
   return SGP_OK;
 }
 
-int sgp_check(sgp_handle *h, const float *d_X, const float *d_W, double *h_stats, void *stream) {
-  if (h == nullptr || d_X == nullptr || d_W == nullptr || h_stats == nullptr) return SGP_ERR_ARG;
+int sgp_colsum(sgp_handle *h, const float *d_A, int include_ring, double *d_out, void *stream) {
+  if (h == nullptr || d_A == nullptr || d_out == nullptr) return SGP_ERR_ARG;
+  const int rc = check_device(h);
+  if (rc != SGP_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  SGP_CUDA_TRY(h, cudaMemsetAsync(h->d_stats, 0, 4 * sizeof(double), st));
-  const unsigned grid = static_cast<unsigned>(h->sm_count * 8);
-  sgp::sgp_scan_kernel<<<grid, 256, 0, st>>>(d_X, h->n, h->d, h->ld, h->d_stats);
-  if (h->tau > 0) sgp::sgp_scan_kernel<<<grid, 256, 0, st>>>(h->ring_x, h->tau * h->n, h->d, h->ld, h->d_stats);
-  sgp::sgp_weight_scan_kernel<<<1, 256, 0, st>>>(d_W, h->n, h->ring_w, h->tau * h->n, h->d_stats);
+  // the statistics of this pass are not wanted: they go to the slots sgp_check clears before it runs
+  sgp::sgp_colsum_kernel<<<column_grid(h), 256, 0, st>>>(d_A, h->n, h->d, h->ld, include_ring ? h->ring_x : nullptr,
+                                                         include_ring ? h->tau * h->n : 0, d_out, nullptr,
+                                                         h->d_stats + kDevStatsCheck);
   SGP_CUDA_TRY(h, cudaGetLastError());
-  double tmp[4];
-  SGP_CUDA_TRY(h, cudaMemcpyAsync(tmp, h->d_stats, sizeof(tmp), cudaMemcpyDeviceToHost, st));
+  return SGP_OK;
+}
+
+int sgp_check(sgp_handle *h, const float *d_X, const float *d_W, const double *d_colsum_ref, double *h_stats,
+              void *stream) {
+  if (h == nullptr || d_X == nullptr || d_W == nullptr || h_stats == nullptr) return SGP_ERR_ARG;
+  int rc = check_device(h);
+  if (rc != SGP_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  rc = enqueue_check(h, d_X, d_W, d_colsum_ref, st);
+  if (rc != SGP_OK) return rc;
+  double tmp[sgp::kStatCount];
+  SGP_CUDA_TRY(h, cudaMemcpyAsync(tmp, h->d_stats + kDevStatsCheck, sizeof(tmp), cudaMemcpyDeviceToHost, st));
   SGP_CUDA_TRY(h, cudaStreamSynchronize(st));
-  h_stats[0] = tmp[2];
-  h_stats[1] = tmp[3];
-  h_stats[2] = tmp[1];
-  h_stats[3] = tmp[0];
+  unsigned status = 0;
+  rc = refresh_status(h, &status);
+  if (rc != SGP_OK) return rc;
+  h_stats[0] = tmp[sgp::kStatSumW];
+  h_stats[1] = tmp[sgp::kStatMinW];
+  h_stats[2] = tmp[sgp::kStatNonFinite];
+  h_stats[3] = tmp[sgp::kStatTotal];
+  h_stats[4] = tmp[sgp::kStatMaxDrift];
+  h_stats[5] = tmp[sgp::kStatMaxRelDrift];
+  h_stats[6] = std::fabs(tmp[sgp::kStatSumW] - static_cast<double>(h->n));
+  h_stats[7] = static_cast<double>(status);
+  if (!(tmp[sgp::kStatMinW] > 0.0)) return SGP_ERR_ZERO_WEIGHT;
+  if (status & kWaitBits) return SGP_ERR_DEVICE;
+  const bool bad = tmp[sgp::kStatNonFinite] > 0.0 || !(h_stats[6] <= 1e-4 * h->n) ||
+                   (d_colsum_ref != nullptr && !(tmp[sgp::kStatMaxRelDrift] <= kColumnDriftTol));
+  return bad ? SGP_ERR_INVARIANT : SGP_OK;
+}
+
+int sgp_get_diagnostics(sgp_handle *h, double *h_param_dev, double *h_consensus, double *h_summary, void *stream) {
+  if (h == nullptr) return SGP_ERR_ARG;
+  if (!h->diag_valid) return SGP_ERR_STATE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  double tmp[2 * SGP_MAX_NODES];
+  const int n = h->n;
+  SGP_CUDA_TRY(h, cudaMemcpyAsync(tmp, h->d_stats + kDevStatsDiag, 2 * static_cast<size_t>(n) * sizeof(double), cudaMemcpyDeviceToHost, st));
+  SGP_CUDA_TRY(h, cudaStreamSynchronize(st));
+  if (h->s_compute != nullptr) SGP_CUDA_TRY(h, cudaStreamSynchronize(h->s_compute));
+  for (int i = 0; i < 2 * n; ++i) tmp[i] = std::sqrt(tmp[i]);
+  for (int part = 0; part < 2; ++part) {
+    double *dst = part == 0 ? h_param_dev : h_consensus;
+    double mean = 0.0, mn = tmp[part * n], mx = tmp[part * n];
+    for (int i = 0; i < n; ++i) {
+      const double v = tmp[part * n + i];
+      if (dst) dst[i] = v;
+      mean += v;
+      mn = std::min(mn, v);
+      mx = std::max(mx, v);
+    }
+    if (h_summary) {
+      h_summary[3 * part + 0] = mean / n;
+      h_summary[3 * part + 1] = mn;
+      h_summary[3 * part + 2] = mx;
+    }
+  }
   return SGP_OK;
 }
 
 int sgp_param_deviation(sgp_handle *h, const float *d_A, double *h_dev, void *stream) {
   if (h == nullptr || d_A == nullptr || h_dev == nullptr) return SGP_ERR_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  double *acc = h->d_stats + 4;
+  double *acc = h->d_stats + kDevStatsDeviation;
   SGP_CUDA_TRY(h, cudaMemsetAsync(acc, 0, static_cast<size_t>(h->n) * sizeof(double), st));
   // tile of n rows x tile_cols columns in shared memory, at most ~64 KB
   int tile_cols = 256;
   while (tile_cols > 32 && static_cast<size_t>(h->n) * tile_cols * 4 > 64 * 1024) tile_cols >>= 1;
   const size_t smem = (static_cast<size_t>(h->n) * tile_cols + tile_cols + h->n) * sizeof(float);
-  if (smem > 48 * 1024)
-    SGP_CUDA_TRY(h, cudaFuncSetAttribute(reinterpret_cast<const void *>(sgp::sgp_deviation_kernel),
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  {
+    sgp::KernelInfo ki;
+    const int rc = sgp::kernel_info(h->dev.device, reinterpret_cast<const void *>(sgp::sgp_deviation_kernel), smem, &ki,
+                                    &h->last_cuda_error);
+    if (rc != SGP_OK) return rc;
+  }
   const int64_t ntiles = (h->d + tile_cols - 1) / tile_cols;
-  const unsigned grid = static_cast<unsigned>(std::min<int64_t>(ntiles, static_cast<int64_t>(h->sm_count) * 2));
+  const unsigned grid = static_cast<unsigned>(std::min<int64_t>(ntiles, static_cast<int64_t>(h->dev.sm_count) * 2));
   sgp::sgp_deviation_kernel<<<grid, 256, smem, st>>>(d_A, h->n, h->d, h->ld, tile_cols, acc);
   SGP_CUDA_TRY(h, cudaGetLastError());
   SGP_CUDA_TRY(h, cudaMemcpyAsync(h_dev, acc, static_cast<size_t>(h->n) * sizeof(double), cudaMemcpyDeviceToHost, st));
@@ -852,6 +844,23 @@ int sgp_set_option(sgp_handle *h, const char *key, int64_t value) {
   } else if (std::strcmp(key, "l2_hint") == 0) {
     if (value > 4) return SGP_ERR_ARG;
     h->opt_l2_hint = value;
+  } else if (std::strcmp(key, "send_period") == 0) {
+    if (value < 1 || value > (1 << 20)) return SGP_ERR_ARG;
+    h->opt_send_period = value;
+  } else if (std::strcmp(key, "diagnostics") == 0) {
+    if (value > 1) return SGP_ERR_ARG;
+    h->opt_diagnostics = value;
+  } else if (std::strcmp(key, "check_steps") == 0) {
+    if (value > 1) return SGP_ERR_ARG;
+    if (value == 1 && h->d_expect == nullptr) {
+      if (check_device(h) != SGP_OK) return SGP_ERR_STATE;
+      if (cudaMalloc(&h->d_expect, static_cast<size_t>(h->d) * sizeof(double)) != cudaSuccess) {
+        (void)cudaGetLastError();
+        h->d_expect = nullptr;
+        return SGP_ERR_ALLOC;
+      }
+    }
+    h->opt_check_steps = value;
   } else {
     return SGP_ERR_ARG;
   }
@@ -868,11 +877,14 @@ int sgp_get_option(const sgp_handle *h, const char *key, int64_t *value) {
   else if (std::strcmp(key, "single_buffer") == 0) *value = h->opt_single_buffer;
   else if (std::strcmp(key, "wait_limit_ms") == 0) *value = h->opt_wait_limit_ms;
   else if (std::strcmp(key, "inject_stall") == 0) *value = h->opt_inject_stall;
-  else if (std::strcmp(key, "last_variant") == 0) *value = h->last_variant;
-  else if (std::strcmp(key, "last_grid") == 0) *value = h->last_grid;
+  else if (std::strcmp(key, "send_period") == 0) *value = h->opt_send_period;
+  else if (std::strcmp(key, "diagnostics") == 0) *value = h->opt_diagnostics;
+  else if (std::strcmp(key, "check_steps") == 0) *value = h->opt_check_steps;
+  else if (std::strcmp(key, "last_variant") == 0) *value = h->last.variant;
+  else if (std::strcmp(key, "last_grid") == 0) *value = h->last.grid;
   else if (std::strcmp(key, "launches") == 0) *value = h->launches;
-  else if (std::strcmp(key, "last_smem") == 0) *value = h->last_smem;
-  else if (std::strcmp(key, "last_tile_cols") == 0) *value = h->last_tile_cols;
+  else if (std::strcmp(key, "last_smem") == 0) *value = h->last.smem;
+  else if (std::strcmp(key, "last_tile_cols") == 0) *value = h->last.tile_cols;
   else return SGP_ERR_ARG;
   return SGP_OK;
 }
@@ -880,8 +892,7 @@ int sgp_get_option(const sgp_handle *h, const char *key, int64_t *value) {
 int sgp_device_status(sgp_handle *h, unsigned *status) {
   if (h == nullptr || status == nullptr) return SGP_ERR_ARG;
   SGP_CUDA_TRY(h, cudaDeviceSynchronize());
-  SGP_CUDA_TRY(h, cudaMemcpy(status, h->d_words + 1, sizeof(unsigned), cudaMemcpyDeviceToHost));
-  return SGP_OK;
+  return refresh_status(h, status);
 }
 
 int sgp_last_cuda_error(const sgp_handle *h) { return h == nullptr ? 0 : h->last_cuda_error; }

@@ -18,10 +18,11 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <cmath>
 #include <mutex>
 
+#include "launch.h"
 #include "sgp.h"
-#include "step_kernels.cuh"
 
 namespace {
 
@@ -66,62 +67,22 @@ int ensure_setup(int *device_out, DeviceSetup *out) {
   return SGP_OK;
 }
 
-using StepKernel = void (*)(const sgp::StepParams, const sgp::ConstTable);
-
-template <int VEC>
-StepKernel pick(bool has_m, bool nesterov, bool has_z) {
-  if (!has_m) return has_z ? sgp::sgp_step_regs_kernel<VEC, sgp::kUpdSgd, true, false>
-                           : sgp::sgp_step_regs_kernel<VEC, sgp::kUpdSgd, false, false>;
-  if (nesterov) return has_z ? sgp::sgp_step_regs_kernel<VEC, sgp::kUpdNesterov, true, false>
-                             : sgp::sgp_step_regs_kernel<VEC, sgp::kUpdNesterov, false, false>;
-  return has_z ? sgp::sgp_step_regs_kernel<VEC, sgp::kUpdHeavyBall, true, false>
-               : sgp::sgp_step_regs_kernel<VEC, sgp::kUpdHeavyBall, false, false>;
-}
-
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-int launch(const DeviceSetup &s, sgp::StepParams p, int vec, int64_t c0, int64_t c1, bool update_w, bool nesterov,
-           cudaStream_t stream) {
+// Same tile sizing, shared-memory budget, grid and kernel-attribute cache as the handle path.
+int launch(const DeviceSetup &s, int dev, sgp::StepParams p, int vec, int64_t c0, int64_t c1, bool update_w, int upd,
+           bool uniform_rows, cudaStream_t stream) {
   p.col_begin = c0;
   p.col_end = c1;
   p.update_w = update_w ? 1 : 0;
-  const size_t table_bytes = (static_cast<size_t>(p.n) + 1 + 2 * static_cast<size_t>(p.nnz)) * 4;
-  p.table_mode = table_bytes <= 40 * 1024 ? 1 : 2;
-  int log2_tv = vec == 4 ? 6 : 8;                         // 256 columns per tile
-  size_t smem = 0;
-  for (;;) {
-    smem = 2 * static_cast<size_t>(p.n) * (size_t{1} << log2_tv) * vec * 4 + 3 * static_cast<size_t>(p.n) * 4 +
-           (p.table_mode < 2 ? table_bytes : 0);
-    if (smem <= 100 * 1024 || log2_tv <= (vec == 4 ? 3 : 5)) break;
-    --log2_tv;
-  }
-  if (smem > static_cast<size_t>(s.smem_optin)) return SGP_ERR_ARG;
-  p.log2_tile_vecs = log2_tv;
-  StepKernel kern = vec == 4 ? pick<4>(p.M != nullptr, nesterov, p.Z != nullptr)
-                             : pick<1>(p.M != nullptr, nesterov, p.Z != nullptr);
-  if (smem > 48 * 1024 &&
-      cudaFuncSetAttribute(reinterpret_cast<const void *>(kern), cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           static_cast<int>(smem)) != cudaSuccess) {
-    (void)cudaGetLastError();
-    return SGP_ERR_CUDA;
-  }
-  // CTAs resident per SM by registers, shared memory and threads: the grid is exactly one wave
-  cudaFuncAttributes fa;
-  if (cudaFuncGetAttributes(&fa, reinterpret_cast<const void *>(kern)) != cudaSuccess) {
-    (void)cudaGetLastError();
-    return SGP_ERR_CUDA;
-  }
-  const int regs_per_cta = ((fa.numRegs + 7) / 8 * 8) * sgp::kThreads;
-  const int resident = std::min({regs_per_cta > 0 ? 65536 / regs_per_cta : 8,
-                                 static_cast<int>((227 * 1024) / (smem + fa.sharedSizeBytes + 1024)),
-                                 2048 / sgp::kThreads});
-  const int64_t tile_cols = (int64_t{1} << log2_tv) * vec;
-  const int64_t ntiles = (c1 - c0 + tile_cols - 1) / tile_cols;
-  const int64_t grid = std::min<int64_t>(ntiles, static_cast<int64_t>(s.sm_count) * std::max(1, resident));
-  static const sgp::ConstTable kNoTable{};
-  kern<<<static_cast<unsigned>(grid), sgp::kThreads, smem, stream>>>(p, kNoTable);
-  if (cudaGetLastError() != cudaSuccess) return SGP_ERR_CUDA;
-  return SGP_OK;
+  sgp::DeviceInfo di;
+  di.device = dev;
+  di.sm_count = s.sm_count;
+  di.smem_optin = s.smem_optin;
+  sgp::RegsOptions opt;
+  if (vec == 4) opt.tile_cols = sgp::regs_tile_cols(p.n, 4 * 1024);
+  sgp::LaunchRecord rec;
+  return sgp::launch_regs(di, p, nullptr, upd, vec, uniform_rows, opt, stream, &rec);
 }
 
 }  // namespace
@@ -137,13 +98,39 @@ extern "C" int sgp_step_static(int n, int64_t d, int64_t ld, const int32_t *h_ro
   for (int i = 0; i < n; ++i)
     if (h_rowptr[i + 1] < h_rowptr[i]) return SGP_ERR_GRAPH;
   for (int64_t e = 0; e < nnz; ++e)
-    if (h_col[e] < 0 || h_col[e] >= n) return SGP_ERR_GRAPH;
+    if (h_col[e] < 0 || h_col[e] >= n || !std::isfinite(h_val[e]) || !(h_val[e] > 0.0f)) return SGP_ERR_GRAPH;
+  {
+    // the same acceptance rule as the schedule compiler: every sender's weights sum to one, self-loops present
+    double colsum[SGP_MAX_NODES] = {0.0};
+    int outdeg[SGP_MAX_NODES] = {0};
+    bool has_self[SGP_MAX_NODES] = {false};
+    for (int i = 0; i < n; ++i)
+      for (int32_t e = h_rowptr[i]; e < h_rowptr[i + 1]; ++e) {
+        const int j = h_col[e];
+        if (e > h_rowptr[i] && h_col[e - 1] >= j) return SGP_ERR_GRAPH;      // senders ascending, no duplicates
+        colsum[j] += static_cast<double>(h_val[e]);
+        ++outdeg[j];
+        if (j == i) has_self[j] = true;
+      }
+    for (int j = 0; j < n; ++j)
+      if (!has_self[j] || std::fabs(colsum[j] - 1.0) > 4.0 * outdeg[j] * std::ldexp(1.0, -24)) return SGP_ERR_GRAPH;
+  }
 
   int dev = 0;
   DeviceSetup s;
   const int rc = ensure_setup(&dev, &s);
   if (rc != SGP_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  {
+    // The table uploads below read the caller's host arrays when they EXECUTE; inside a stream capture that would
+    // be at every replay, long after this call returned.  Captured calls are therefore refused.
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cs) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return SGP_ERR_CUDA;
+    }
+    if (cs != cudaStreamCaptureStatusNone) return SGP_ERR_STATE;
+  }
 
   unsigned *words = reinterpret_cast<unsigned *>(s.scratch);
   int32_t *t_rowptr = reinterpret_cast<int32_t *>(s.scratch + kWordsBytes);
@@ -176,13 +163,22 @@ extern "C" int sgp_step_static(int n, int64_t d, int64_t ld, const int32_t *h_ro
   p.ticket = words;
   p.status = words + 1;
 
+  // every receiver alike (complete graph): the mix is one shared column sum, as in the handle path
+  bool uniform_rows = n > 1;
+  for (int i = 1; i < n && uniform_rows; ++i) {
+    const int32_t len = h_rowptr[1] - h_rowptr[0], b = h_rowptr[i];
+    if (h_rowptr[i + 1] - b != len) uniform_rows = false;
+    for (int32_t e = 0; e < len && uniform_rows; ++e)
+      if (h_col[b + e] != h_col[e] || h_val[b + e] != h_val[e]) uniform_rows = false;
+  }
+  const int upd = momentum == 0.0f ? sgp::kUpdSgd : (nesterov != 0 ? sgp::kUpdNesterov : sgp::kUpdHeavyBall);
   const bool vec_ok = aligned16(d_X) && aligned16(d_G) && (p.M == nullptr || aligned16(p.M)) &&
                       (d_Z == nullptr || aligned16(d_Z)) && (ld % 4 == 0);
   const int64_t vec_end = vec_ok ? (d & ~int64_t{3}) : 0;
   if (vec_end > 0) {
-    const int r = launch(s, p, 4, 0, vec_end, vec_end == d, nesterov != 0, st);
+    const int r = launch(s, dev, p, 4, 0, vec_end, vec_end == d, upd, uniform_rows, st);
     if (r != SGP_OK) return r;
   }
-  if (vec_end < d) return launch(s, p, 1, vec_end, d, true, nesterov != 0, st);
+  if (vec_end < d) return launch(s, dev, p, 1, vec_end, d, true, upd, uniform_rows, st);
   return SGP_OK;
 }

@@ -1,0 +1,200 @@
+// Register-staged fused SGP step kernel: every thread keeps kItemsPerThread (row, vector-column) items in
+// flight, writes x^(k+1/2) into a shared tile, one barrier, then gathers its receivers' rows from the tile
+// (Alg. 1 lines 4-8, Alg. 3 lines 4-5, Alg. 2 with the delayed-message ring).  The tile is double-buffered so
+// one barrier per tile suffices; large n uses one tile and two barriers so that row segments stay long.
+#pragma once
+#include "step_common.cuh"
+
+namespace sgp {
+
+template <int VEC, int UPD, bool HAS_Z, bool HAS_RING, bool DIAG>
+__global__ void __launch_bounds__(kThreads, 2)
+sgp_step_regs_kernel(const __grid_constant__ StepParams p, const __grid_constant__ ConstTable ct) {
+  using V = typename VecT<VEC>::type;
+  constexpr bool HAS_M = UpdTraits<UPD>::kHasM;
+  constexpr bool HAS_V = UpdTraits<UPD>::kHasV;
+  constexpr int kItemsPerThread = UpdTraits<UPD>::kItems;
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  const int n = p.n;
+  const int tv = 1 << p.log2_tile_vecs;
+  const int tile_items = n * tv;
+  V *H0 = reinterpret_cast<V *>(smem_raw);
+  V *H1 = p.single_buffer ? H0 : H0 + tile_items;
+  V *partial = H0 + (p.single_buffer ? 1 : 2) * tile_items;          // uniform_parts x tv vectors (uniform rows only)
+  float *scratch = reinterpret_cast<float *>(partial + p.uniform_parts * tv);
+  const CtaTables tab = cta_prologue<HAS_RING>(p, ct, scratch, kThreads);
+  constexpr bool diag = DIAG;      // fused diagnostics: a separate instantiation, so the plain step pays nothing
+  // The diagnostics' scratch sits after the weights and, when it was copied, the table.  Its pointers are
+  // re-derived where they are used (diagnostics only) instead of being kept live through the hot loop.
+  auto diag_ds = [&]() {
+    unsigned char *after = smem_raw + (static_cast<size_t>(p.single_buffer ? 1 : 2) * tile_items + static_cast<size_t>(p.uniform_parts) * tv) * sizeof(V) +
+                           3 * static_cast<size_t>(n) * 4 + (p.table_mode < 2 ? (static_cast<size_t>(n) + 1 + 2 * static_cast<size_t>(p.nnz)) * 4 : 0);
+    return diag_scratch<V>(after, n, tv, p.diag_parts);
+  };
+  if (diag) {
+    const DiagScratch<V> ds = diag_ds();
+    for (int i = threadIdx.x; i < 2 * n; i += kThreads) ds.rowacc[i] = 0.0;
+    __syncthreads();
+  }
+
+  const int64_t ld = p.ld;
+  const int64_t ncols = p.col_end - p.col_begin;
+  const int64_t tile_cols = static_cast<int64_t>(tv) * VEC;
+  const int64_t ntiles = (ncols + tile_cols - 1) / tile_cols;
+  int buf = 0;
+  // The tile is worked off in batches of at most kItemsPerThread items per thread; the batches are made
+  // equal (e.g. 1280 items: 3 + 2 per thread, not 4 + 1) so that no batch runs with few loads in flight.
+  const int batches = (tile_items + kThreads * kItemsPerThread - 1) / (kThreads * kItemsPerThread);
+  const int q_max = ((tile_items + batches - 1) / batches + kThreads - 1) / kThreads;   // items per thread per batch
+  const int batch_items = q_max * kThreads;
+
+  for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+    const int64_t col0 = p.col_begin + tile * tile_cols;
+    V *H = buf ? H1 : H0;
+    // ---- phase 1: local update, all batches of this tile
+    for (int base = 0; base < tile_items; base += batch_items) {
+      V x[kItemsPerThread], g[kItemsPerThread], u[kItemsPerThread], vv[kItemsPerThread];
+      bool ok[kItemsPerThread];
+      int64_t off[kItemsPerThread];
+#pragma unroll
+      for (int q = 0; q < kItemsPerThread; ++q) {
+        const int item = base + q * kThreads + threadIdx.x;
+        const int row = item >> p.log2_tile_vecs;
+        const int c = item & (tv - 1);
+        const int64_t col = col0 + static_cast<int64_t>(c) * VEC;
+        ok[q] = (q < q_max) && (item < tile_items) && (col < p.col_end);
+        off[q] = static_cast<int64_t>(row) * ld + col;
+        if (ok[q]) ok[q] = SGP_BOUNDS_OK(p, row < n && col >= 0 && col + VEC <= ld);
+      }
+#pragma unroll
+      for (int q = 0; q < kItemsPerThread; ++q) {
+        if (ok[q]) {
+          x[q] = ld_inplace(reinterpret_cast<const V *>(p.X + off[q]));
+          g[q] = ld_stream(reinterpret_cast<const V *>(p.G + off[q]));
+          if (HAS_M) u[q] = ld_inplace(reinterpret_cast<const V *>(p.M + off[q]));
+          if (HAS_V) vv[q] = ld_inplace(reinterpret_cast<const V *>(p.V + off[q]));
+        }
+      }
+#pragma unroll
+      for (int q = 0; q < kItemsPerThread; ++q) {
+        const int item = base + q * kThreads + threadIdx.x;
+        if (ok[q]) {
+          const V h = local_update<UPD, V>(x[q], g[q], u[q], vv[q], p);
+          if (HAS_M) st_stream(reinterpret_cast<V *>(p.M + off[q]), u[q]);
+          if (HAS_V) st_stream(reinterpret_cast<V *>(p.V + off[q]), vv[q]);
+          H[item] = h;
+        } else if (q < q_max && item < tile_items) {
+          H[item] = vzero<V>();
+        }
+      }
+    }
+    __syncthreads();
+    if (diag)
+      diag_column_means<VEC, HAS_RING, V>(p, H, static_cast<const V *>(nullptr), col0, diag_ds(), threadIdx.x, kThreads,
+                                          [] { __syncthreads(); });
+    // ---- phase 2, all receivers alike (complete graph): one weighted column sum, shared by every row
+    if (!HAS_RING && p.uniform_parts > 0) {
+      const int parts = p.uniform_parts;
+      const int e0 = tab.rowptr[0], e1 = tab.rowptr[1];
+      for (int idx = threadIdx.x; idx < tv * parts; idx += kThreads) {
+        const int c = idx & (tv - 1), part = idx >> p.log2_tile_vecs;
+        V acc = vzero<V>();
+        for (int e = e0 + part; e < e1; e += parts) {
+          const int j = tab.col[e];
+          if (SGP_BOUNDS_OK(p, j >= 0 && j < n)) acc = vfma(tab.val[e], H[(j << p.log2_tile_vecs) + c], acc);
+        }
+        partial[idx] = acc;
+      }
+      __syncthreads();
+      for (int it0 = 0; it0 < tile_items; it0 += kThreads) {
+        const int item = it0 + threadIdx.x;
+        const int row = item >> p.log2_tile_vecs;
+        const int c = item & (tv - 1);
+        const int64_t col = col0 + static_cast<int64_t>(c) * VEC;
+        float dq = 0.f, cq = 0.f;
+        if (item < tile_items && col < p.col_end) {
+          const int64_t o = static_cast<int64_t>(row) * ld + col;
+          V acc = partial[c];
+          for (int part = 1; part < parts; ++part) acc = vadd(acc, partial[part * tv + c]);
+          const V z = vmul(tab.inv_w[row], acc);
+          st_stream(reinterpret_cast<V *>(p.X + o), acc);
+          if (HAS_Z) st_stream(reinterpret_cast<V *>(p.Z + o), z);
+          if (diag) {
+            const DiagScratch<V> ds = diag_ds();
+            dq = vsq(vsub(H[item], ds.mean_h[c]));
+            cq = vsq(vsub(z, ds.mean_x[c]));
+          }
+        }
+        if (diag) diag_accumulate(dq, cq, row, n, tv < 32 ? tv : 32, diag_ds().rowacc, item < tile_items);
+      }
+      buf ^= 1;
+      if (p.single_buffer || diag) __syncthreads();
+      continue;
+    }
+    // ---- phase 2: gather-mix over the step's in-neighbour lists, ring exchange, de-bias
+    for (int base = 0; base < tile_items; base += batch_items) {
+      V ring_in[kItemsPerThread];
+      if (HAS_RING) {
+#pragma unroll
+        for (int q = 0; q < kItemsPerThread; ++q) {
+          const int item = base + q * kThreads + threadIdx.x;
+          const int row = item >> p.log2_tile_vecs;
+          const int c = item & (tv - 1);
+          const int64_t col = col0 + static_cast<int64_t>(c) * VEC;
+          if (q < q_max && item < tile_items && col < p.col_end)
+            ring_in[q] = ld_inplace(reinterpret_cast<const V *>(p.ring_x + static_cast<int64_t>(row) * ld + col));
+        }
+      }
+#pragma unroll
+      for (int q = 0; q < kItemsPerThread; ++q) {
+        const int item = base + q * kThreads + threadIdx.x;
+        const int row = item >> p.log2_tile_vecs;
+        const int c = item & (tv - 1);
+        const int64_t col = col0 + static_cast<int64_t>(c) * VEC;
+        float dq = 0.f, cq = 0.f;
+        if (q < q_max && item < tile_items && col < p.col_end) {
+          const int64_t o = static_cast<int64_t>(row) * ld + col;
+          V acc = vzero<V>(), offd = vzero<V>();
+          const int e1 = tab.rowptr[row + 1];
+          for (int e = tab.rowptr[row]; e < e1; ++e) {
+            const int j = tab.col[e];
+            if (!SGP_BOUNDS_OK(p, j >= 0 && j < n)) continue;
+            const float pv = tab.val[e];
+            const V hj = H[(j << p.log2_tile_vecs) + c];
+            if (HAS_RING && j != row) offd = vfma(pv, hj, offd);
+            else acc = vfma(pv, hj, acc);
+          }
+          if (HAS_RING) {
+            acc = vadd(acc, ring_in[q]);
+            st_stream(reinterpret_cast<V *>(p.ring_x + o), offd);
+          }
+          const V z = vmul(tab.inv_w[row], acc);
+          st_stream(reinterpret_cast<V *>(p.X + o), acc);
+          if (HAS_Z) st_stream(reinterpret_cast<V *>(p.Z + o), z);
+          if (diag) {
+            const DiagScratch<V> ds = diag_ds();
+            dq = vsq(vsub(H[item], ds.mean_h[c]));
+            cq = vsq(vsub(z, ds.mean_x[c]));
+          }
+        }
+        if (diag && q < q_max) diag_accumulate(dq, cq, row, n, tv < 32 ? tv : 32, diag_ds().rowacc, item < tile_items);
+      }
+    }
+    buf ^= 1;
+    if (p.single_buffer || diag) __syncthreads();   // the only tile (or the column means) is about to be overwritten
+  }
+  if (diag) {
+    __syncthreads();
+    const DiagScratch<V> ds = diag_ds();
+    for (int i = threadIdx.x; i < 2 * n; i += kThreads)
+      if (ds.rowacc[i] != 0.0) atomicAdd(p.diag + i, ds.rowacc[i]);
+  }
+}
+
+using RegsKernel = void (*)(const StepParams, const ConstTable);
+// The instantiation for (vector width 4 or 1, optimiser, Z written, delay ring, fused diagnostics); the kernels are
+// spread over several translation units so that they compile in parallel.
+RegsKernel regs_kernel(int vec, int upd, bool has_z, bool has_ring, bool diag);
+template <int VEC, bool DIAG> RegsKernel regs_kernel_of(int upd, bool has_z, bool has_ring);
+
+}  // namespace sgp

@@ -13,8 +13,8 @@ def oracle_P_of_k(w):
     """Dense mixing matrices of a workload, from the oracle's own generator."""
     if w.graph == "exp":
         return lambda k: osched.mixing_matrix("exp", w.n, k, peers=w.peers)
-    if w.graph == "complete":
-        return lambda k: osched.mixing_matrix("complete", w.n, k)
+    if w.graph in ("complete", "bipartite"):
+        return lambda k: osched.mixing_matrix(w.graph, w.n, k)
     if w.graph == "random":
         return lambda k: osched.mixing_matrix("random", w.n, k, seed=w.seed, max_outdeg=w.max_outdeg,
                                               num_steps=w.num_steps)

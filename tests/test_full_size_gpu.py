@@ -60,10 +60,22 @@ def _run_full(binding, inputs, w, K, ld_align=256):
             inputs.gradient(w, k, G)
             for i, (a, b) in enumerate(wins):
                 grads[i].append(G[:, a:b].cpu().numpy().copy())
+            if k == K - 1:
+                # per-column conservation over ALL d columns for the last step (Sec. 2: 1^T P = 1^T): what the
+                # columns of X plus ring must sum to follows from column sums of X, G and the new momentum
+                before_all, before_x = h.colsum(X, include_ring=True), h.colsum(X)
             h.step(X, W, M, G, Z, k, w.lr, w.momentum, w.weight_decay, w.nesterov)
+        s = h.colsum(G) + w.weight_decay * before_x
+        if M is not None:
+            s = w.momentum * h.colsum(M) + s if w.nesterov else h.colsum(M)
+        ref = (before_all - w.lr * s).contiguous()
+        del before_all, before_x, s
         torch.cuda.synchronize()
         assert h.device_status() == 0
-        sum_w, min_w, nonfinite, _ = h.check(X, W)
+        stats = h.check(X, W, colsum_ref=ref)
+        sum_w, min_w, nonfinite = stats["sum_w"], stats["min_w"], stats["nonfinite"]
+        del ref
+    assert stats["code"] == 0 and stats["max_colsum_rel_drift"] <= 2e-6, stats
     assert abs(sum_w - n) <= 1e-4 * n and min_w > 0 and nonfinite == 0
     assert torch.isfinite(Z).all().item()
     for i, (a, b) in enumerate(wins):
@@ -118,6 +130,8 @@ def test_transformer_adam_full_size(binding, inputs):
             inputs.gradient(w, k, G)
             for i, (a, b) in enumerate(wins):
                 grads[i].append(G[:, a:b].cpu().numpy().copy())
+            if k == K - 1:
+                h.set_option("check_steps", 1)     # the last step is bracketed by the per-column conservation check
             h.step_adam(X, W, M1, M2, G, Z, k, k + 1, w.lr, w.beta1, w.beta2, w.adam_eps, 0.0)
         torch.cuda.synchronize()
         assert h.device_status() == 0
@@ -140,11 +154,10 @@ def test_tau_full_size_mass_conservation(binding, inputs):
     Z = torch.empty_like(X)
     G = torch.zeros_like(X)
     W = torch.ones(n, device=DEV)
-    before = X.sum(dtype=torch.float64).item()
-    scale = X.abs().sum(dtype=torch.float64).item()
     with binding.Sgp(n, d, graph_desc(w, binding), tau=2) as h:
+        ref = h.colsum(X, include_ring=True).clone()
         for k in range(7):
             h.step(X, W, None, G, Z, k, w.lr, 0.0, 0.0, True)
-        sum_w, min_w, nonfinite, total = h.check(X, W)
-    assert abs(sum_w - n) <= 1e-4 * n and nonfinite == 0
-    assert abs(total - before) <= 1e-5 * scale
+        stats = h.check(X, W, colsum_ref=ref)
+    assert stats["code"] == 0 and stats["max_colsum_rel_drift"] <= 2e-6, stats
+    assert abs(stats["sum_w"] - n) <= 1e-4 * n and stats["nonfinite"] == 0

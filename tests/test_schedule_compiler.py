@@ -57,6 +57,21 @@ def test_random_outdeg_bit_exact(binding, n, seed, max_outdeg, steps):
                                                      num_steps=steps))
 
 
+@pytest.mark.parametrize("n", [2, 4, 6, 8, 10, 16, 32, 64, 100, 256])
+def test_bipartite_exp_bit_exact(binding, n):
+    sched = binding.Schedule(n, binding.GraphDesc.bipartite_exp())
+    assert sched.period == S.schedule_period("bipartite", n)
+    for k in range(2 * sched.period + 1):
+        _assert_slot_equal(sched, k, S.mixing_matrix("bipartite", n, k))
+
+
+@pytest.mark.parametrize("n", [1, 3, 7, 255])
+def test_bipartite_exp_needs_an_even_node_count(binding, n):
+    with pytest.raises(binding.SgpError) as e:
+        binding.Schedule(n, binding.GraphDesc.bipartite_exp())
+    assert e.value.code == binding.SGP_ERR_ARG
+
+
 def _four_node_edges():
     rows = read_golden("four_node_update_equations.txt")
     recv = [int(r[0]) for r in rows]
