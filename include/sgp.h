@@ -324,6 +324,75 @@ int sgp_step_static(int n, int64_t d, int64_t ld, const int32_t *h_rowptr, const
                     const float *h_val, int64_t nnz, float *d_X, float *d_W, float *d_M, const float *d_G,
                     float *d_Z, float lr, float momentum, float weight_decay, int nesterov, void *stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * One node per GPU (App. C "Implementation Details": every node sends (p x, p w) to its out-neighbours and adds
+ * what it receives; Sec. 3 "Overlapping communication and computation", Alg. 2).  Rank r of `world` = n nodes
+ * holds ONE row of every array: x, m, g, z are d floats, w is one float, all DEVICE memory of the caller.
+ * The step is split where data crosses between nodes:
+ *     update : h = x - lr * s, written UNWEIGHTED with w into a message slot in this GPU's memory (the "send")
+ *     mix    : x' = sum_j p_ij h_j, w' = sum_j p_ij w_j, z = x' / w', reading every in-neighbour's slot directly
+ *              from that GPU's memory with plain loads over NVLink (peer pointers): pull and mix are one kernel;
+ *              the receiver applies p_ij, so all out-neighbours of a node read the same slot
+ *     tau >= 1 : the messages consumed at step k were published at step k - tau, so update + pull + mix are ONE
+ *              kernel per step (sgp_rank_step_overlap) and the exchange never waits.
+ * Results are bit-identical to sgp_step on the stacked n x d arrays (same CSR order, same FMA chain).
+ *
+ * Synchronisation is the caller's (one barrier per step across the ranks, e.g. an all-reduce of one element on the
+ * step's stream): tau == 0: update, BARRIER, mix; tau >= 1: step_overlap, BARRIER.  No kernel of this library
+ * waits on another GPU.  A rank keeps tau + 2 message slots: a slot is rewritten tau + 2 steps after it was
+ * published, when every reader has passed at least one barrier since its read.
+ * Not supported here: send_period, Adam, in-degree above SGP_RANK_MAX_SOURCES (SGP_ERR_ARG; the complete graph
+ * is what an all-reduce is for).
+ * ------------------------------------------------------------------------------------------- */
+typedef struct sgp_rank sgp_rank;
+#define SGP_RANK_MAX_SOURCES 32
+#define SGP_IPC_HANDLE_BYTES 64
+
+/* What rank `rank` does at step k (HOST only, needs no GPU): which slot it publishes into, which slot of its
+ * in-neighbours it reads, its own weight p_ii^(k), and the in-neighbours with the weights p_ij it applies, in the
+ * order of the sum.  tau == 0: the list is row `rank` of P^(k), self included at self_pos, read_slot == write_slot.
+ * tau >= 1: the list is row `rank` of P^(k - tau) without the diagonal (empty while k < tau: nothing has
+ * arrived yet), self_pos = -1, and the node's own half step enters with self_weight. */
+typedef struct sgp_rank_plan_t {
+  int32_t write_slot, read_slot;
+  float   self_weight;
+  int32_t self_pos;
+  int32_t count;
+  int32_t sender[SGP_RANK_MAX_SOURCES];
+  float   weight[SGP_RANK_MAX_SOURCES];
+} sgp_rank_plan_t;
+int sgp_rank_plan(const sgp_schedule *s, int rank, int64_t k, int tau, sgp_rank_plan_t *out);
+
+/* Creates rank `rank` of `world` on the current device: compiles the schedule for n = world nodes and allocates
+ * and zeroes (tau + 2) message slots of d (+ padding) floats.  Synchronises. */
+int sgp_rank_create(sgp_rank **out, int rank, int world, int64_t d, const sgp_graph_desc *g, int tau, unsigned flags);
+int sgp_rank_destroy(sgp_rank *r);
+int sgp_rank_get_schedule(const sgp_rank *r, const sgp_schedule **s);
+/* The rank's message slots: one device allocation of `bytes` bytes.  Other ranks need its address in THEIR
+ * process: the same pointer inside one process, or sgp_ipc_export here + sgp_ipc_open there. */
+int sgp_rank_message_block(sgp_rank *r, void **d_block, size_t *bytes);
+/* d_peer_blocks[j] (HOST array of `world` device pointers valid in this process; entry [rank] is ignored, entries
+ * of ranks this node never receives from may be NULL): where rank j's message block is mapped. */
+int sgp_rank_set_peers(sgp_rank *r, void *const *d_peer_blocks);
+/* tau == 0, first half: publishes (h, w) of step k; m updated in place; x untouched.  Asynchronous. */
+int sgp_rank_update(sgp_rank *r, const float *d_x, float *d_w, float *d_m, const float *d_g, int64_t k, float lr,
+                    float momentum, float weight_decay, int nesterov, void *stream);
+/* tau == 0, second half, after every in-neighbour's update of step k is complete: pull + mix + de-bias; writes x,
+ * w, z (d_z may be NULL).  SGP_ERR_STATE if tau != 0 or a needed peer block was never set.  Asynchronous. */
+int sgp_rank_mix(sgp_rank *r, float *d_x, float *d_w, float *d_z, int64_t k, void *stream);
+/* tau >= 1: the whole step k in one kernel (Alg. 2).  Steps must be presented in order.  SGP_ERR_STATE if
+ * tau == 0.  Asynchronous. */
+int sgp_rank_step_overlap(sgp_rank *r, float *d_x, float *d_w, float *d_m, const float *d_g, float *d_z, int64_t k,
+                          float lr, float momentum, float weight_decay, int nesterov, void *stream);
+/* SGP_STATUS_ZERO_WEIGHT is the only bit this mode sets.  Synchronises. */
+int sgp_rank_device_status(sgp_rank *r, unsigned *status);
+/* Thin wrappers of the CUDA IPC calls for callers without a CUDA binding: `handle` is SGP_IPC_HANDLE_BYTES bytes of
+ * HOST memory to ship to the other process by any means; sgp_ipc_open maps the exporter's allocation into this
+ * process (peer access is enabled as needed) and sgp_ipc_close unmaps it. */
+int sgp_ipc_export(const void *d_ptr, unsigned char *handle);
+int sgp_ipc_open(const unsigned char *handle, void **d_ptr);
+int sgp_ipc_close(void *d_ptr);
+
 /* Reads the handle's device status word (SGP_STATUS_* bits; 0 = nothing ever went wrong).  Once a wait bit or
  * the zero-weight bit has been seen by a synchronising call (this one, sgp_check, sgp_step_host), later
  * sgp_step / sgp_step_adam calls return SGP_ERR_DEVICE / SGP_ERR_ZERO_WEIGHT until sgp_reset, which clears the

@@ -31,7 +31,12 @@ EXPORTS = [
     "sgp_ring_export", "sgp_ring_import", "sgp_check", "sgp_set_option", "sgp_get_option", "sgp_device_status",
     "sgp_last_cuda_error", "sgp_strerror", "sgp_version", "sgp_step_static",
     "sgp_step_adam", "sgp_param_deviation", "sgp_set_graph", "sgp_colsum", "sgp_get_diagnostics",
+    "sgp_rank_plan", "sgp_rank_create", "sgp_rank_destroy", "sgp_rank_get_schedule", "sgp_rank_message_block",
+    "sgp_rank_set_peers", "sgp_rank_update", "sgp_rank_mix", "sgp_rank_step_overlap", "sgp_rank_device_status",
+    "sgp_ipc_export", "sgp_ipc_open", "sgp_ipc_close",
 ]
+SGP_RANK_MAX_SOURCES = 32
+SGP_IPC_HANDLE_BYTES = 64
 
 
 class SgpError(RuntimeError):
@@ -48,6 +53,11 @@ class sgp_graph_desc(C.Structure):
         ("edge_receiver", C.POINTER(C.c_int32)), ("edge_weight", C.POINTER(C.c_float)),
         ("num_edges", C.c_int64),
     ]
+
+
+class sgp_rank_plan_t(C.Structure):
+    _fields_ = [("write_slot", C.c_int32), ("read_slot", C.c_int32), ("self_weight", C.c_float),
+                ("self_pos", C.c_int32), ("count", C.c_int32), ("sender", C.c_int32 * 32), ("weight", C.c_float * 32)]
 
 
 def _load() -> C.CDLL:
@@ -83,6 +93,19 @@ def _load() -> C.CDLL:
         "sgp_device_status": [vp, C.POINTER(C.c_uint)],
         "sgp_last_cuda_error": [vp],
         "sgp_version": [],
+        "sgp_rank_plan": [vp, i32, i64, i32, C.POINTER(sgp_rank_plan_t)],
+        "sgp_rank_create": [C.POINTER(vp), i32, i32, i64, C.POINTER(sgp_graph_desc), i32, C.c_uint],
+        "sgp_rank_destroy": [vp],
+        "sgp_rank_get_schedule": [vp, C.POINTER(vp)],
+        "sgp_rank_message_block": [vp, C.POINTER(vp), C.POINTER(C.c_size_t)],
+        "sgp_rank_set_peers": [vp, C.POINTER(vp)],
+        "sgp_rank_update": [vp, vp, vp, vp, vp, i64, f32, f32, f32, i32, vp],
+        "sgp_rank_mix": [vp, vp, vp, vp, i64, vp],
+        "sgp_rank_step_overlap": [vp, vp, vp, vp, vp, vp, i64, f32, f32, f32, i32, vp],
+        "sgp_rank_device_status": [vp, C.POINTER(C.c_uint)],
+        "sgp_ipc_export": [vp, C.c_char_p],
+        "sgp_ipc_open": [C.c_char_p, C.POINTER(vp)],
+        "sgp_ipc_close": [vp],
         "sgp_step_static": [i32, i64, i64, vp, vp, vp, i64, vp, vp, vp, vp, vp, f32, f32, f32, i32, vp],
     }
     for name, args in sig.items():
@@ -178,6 +201,15 @@ class _ScheduleView:
         _check(_lib.sgp_schedule_get(self._ptr, k, rowptr.ctypes.data, col.ctypes.data, val.ctypes.data, nnz,
                                      C.byref(out)), "sgp_schedule_get")
         return rowptr, col[:nnz], val[:nnz]
+
+
+def rank_plan(schedule: "_ScheduleView", rank: int, k: int, tau: int) -> dict:
+    """sgp_rank_plan (host only): what `rank` publishes and pulls at step k in the one-node-per-GPU mode."""
+    out = sgp_rank_plan_t()
+    _check(_lib.sgp_rank_plan(schedule._ptr, rank, k, tau, C.byref(out)), "sgp_rank_plan")
+    return dict(write_slot=out.write_slot, read_slot=out.read_slot, self_weight=np.float32(out.self_weight),
+                self_pos=out.self_pos, senders=[out.sender[e] for e in range(out.count)],
+                weights=np.array([out.weight[e] for e in range(out.count)], dtype=np.float32))
 
 
 class Schedule(_ScheduleView):
@@ -348,6 +380,76 @@ class Sgp:
 
     def last_cuda_error(self) -> int:
         return _lib.sgp_last_cuda_error(self._h)
+
+
+class SgpRank:
+    """sgp_rank_*: one node of the one-node-per-GPU mode.  x, m, g, z are 1-D float32 CUDA tensors of d entries,
+    w is a float32 CUDA tensor of one entry.  Marshalling only; see rowshard.py for the orchestration."""
+
+    def __init__(self, rank: int, world: int, d: int, graph: GraphDesc, tau: int = 0, flags: int = 0):
+        self.rank, self.world, self.d, self.tau = rank, world, d, tau
+        self._h = C.c_void_p()
+        _check(_lib.sgp_rank_create(C.byref(self._h), rank, world, d, C.byref(graph.c), tau, flags), "sgp_rank_create")
+
+    def close(self):
+        if getattr(self, "_h", None) and _lib is not None:
+            _lib.sgp_rank_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        self.close()
+
+    @property
+    def schedule(self) -> _ScheduleView:
+        p = C.c_void_p()
+        _check(_lib.sgp_rank_get_schedule(self._h, C.byref(p)), "sgp_rank_get_schedule")
+        return _ScheduleView(p, self.world)
+
+    def message_block(self):
+        """(device pointer, bytes) of this rank's message slots."""
+        ptr, size = C.c_void_p(), C.c_size_t()
+        _check(_lib.sgp_rank_message_block(self._h, C.byref(ptr), C.byref(size)), "sgp_rank_message_block")
+        return ptr.value, size.value
+
+    def set_peers(self, pointers) -> None:
+        """pointers[j]: device address (int or None) of rank j's message block in this process."""
+        arr = (C.c_void_p * self.world)(*[C.c_void_p(p) if p else None for p in pointers])
+        _check(_lib.sgp_rank_set_peers(self._h, arr), "sgp_rank_set_peers")
+
+    def update(self, x, w, m, g, k: int, lr: float, momentum: float = 0.0, weight_decay: float = 0.0,
+               nesterov: bool = True, stream=None) -> None:
+        _check(_lib.sgp_rank_update(self._h, _ptr(x), _ptr(w), _ptr(m), _ptr(g), k, lr, momentum, weight_decay,
+                                    int(bool(nesterov)), _stream_ptr(stream)), "sgp_rank_update")
+
+    def mix(self, x, w, z, k: int, stream=None) -> None:
+        _check(_lib.sgp_rank_mix(self._h, _ptr(x), _ptr(w), _ptr(z), k, _stream_ptr(stream)), "sgp_rank_mix")
+
+    def step_overlap(self, x, w, m, g, z, k: int, lr: float, momentum: float = 0.0, weight_decay: float = 0.0,
+                     nesterov: bool = True, stream=None) -> None:
+        _check(_lib.sgp_rank_step_overlap(self._h, _ptr(x), _ptr(w), _ptr(m), _ptr(g), _ptr(z), k, lr, momentum,
+                                          weight_decay, int(bool(nesterov)), _stream_ptr(stream)),
+               "sgp_rank_step_overlap")
+
+    def device_status(self) -> int:
+        v = C.c_uint()
+        _check(_lib.sgp_rank_device_status(self._h, C.byref(v)), "sgp_rank_device_status")
+        return v.value
+
+
+def ipc_export(device_ptr: int) -> bytes:
+    buf = C.create_string_buffer(SGP_IPC_HANDLE_BYTES)
+    _check(_lib.sgp_ipc_export(C.c_void_p(device_ptr), buf), "sgp_ipc_export")
+    return buf.raw
+
+
+def ipc_open(handle: bytes) -> int:
+    ptr = C.c_void_p()
+    _check(_lib.sgp_ipc_open(handle, C.byref(ptr)), "sgp_ipc_open")
+    return ptr.value
+
+
+def ipc_close(device_ptr: int) -> None:
+    _check(_lib.sgp_ipc_close(C.c_void_p(device_ptr)), "sgp_ipc_close")
 
 
 def step_static(n: int, d: int, ld: int, rowptr, col, val, X, W, M, G, Z, lr: float, momentum: float = 0.0,

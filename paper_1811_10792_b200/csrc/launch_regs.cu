@@ -90,6 +90,7 @@ int launch_regs(const DeviceInfo &dev, StepParams p, const ConstTable *ct, int u
   int64_t tv = int64_t{1} << floor_log2(std::max<int64_t>(1, kThreads * 4 / n));
   if (opt.tile_cols > 0) tv = int64_t{1} << floor_log2(std::max<int64_t>(1, opt.tile_cols / vec));
   tv = std::max<int64_t>(tv, min_tv);
+  if (p.diag != nullptr) tv = std::min<int64_t>(tv, 256);   // diagnostics: a thread owns one column of every tile
   // short rows: narrower tiles until there is about a tile per SM (launch-latency regime)
   if (!opt.tile_cols_forced)
     while (tv > min_tv && tv * vec > 128 && (ncols + tv * vec - 1) / (tv * vec) < dev.sm_count) tv >>= 1;
@@ -99,15 +100,17 @@ int launch_regs(const DeviceInfo &dev, StepParams p, const ConstTable *ct, int u
   const bool uniform = !has_ring && uniform_rows;
   // large n: one exchange tile (two barriers per tile) so that the row segments can stay twice as long
   p.single_buffer = opt.single_buffer == 1 ? 1 : (opt.single_buffer == 2 ? 0 : (auto_single_buffer(n) ? 1 : 0));
+  // diagnostics add up to 32 KB of scratch: one exchange tile then keeps the CTA's footprint (and with it the
+  // share of the SM left to the L1) where it was (tau = 1, n = 32: 96 KB per CTA ran at 0.67, 64 KB does not)
+  if (p.diag != nullptr && opt.single_buffer == 0) p.single_buffer = 1;
   size_t smem = 0;
   for (;;) {
     const int parts = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(8, kThreads / tv)));
     p.uniform_parts = uniform ? parts : 0;
-    p.diag_parts = parts;
     smem = (p.single_buffer ? 1 : 2) * static_cast<size_t>(n) * tv * vec * 4 + 3 * static_cast<size_t>(n) * 4 +
            static_cast<size_t>(p.uniform_parts) * tv * vec * 4 + (p.table_mode < 2 ? table_bytes : 0);
     if (p.diag != nullptr)
-      smem += vec == 4 ? diag_scratch_bytes<float4>(n, static_cast<int>(tv), parts) : diag_scratch_bytes<float>(n, static_cast<int>(tv), parts);
+      smem += vec == 4 ? diag_scratch_bytes<float4>(n, static_cast<int>(tv), has_ring) : diag_scratch_bytes<float>(n, static_cast<int>(tv), has_ring);
     if (smem <= 110 * 1024 || tv <= min_tv) break;
     tv >>= 1;
   }

@@ -28,6 +28,7 @@ int launch_tma(const DeviceInfo &dev, StepParams p, const ConstTable *ct, int up
   const int arrays = 2 + (has_m ? 1 : 0) + (has_v ? 1 : 0) + (has_ring ? 1 : 0);
   int64_t tv = int64_t{1} << floor_log2(std::max<int64_t>(1, (opt.tile_cols > 0 ? opt.tile_cols : 256) / 4));
   tv = std::max<int64_t>(tv, 8);
+  if (p.diag != nullptr) tv = std::min<int64_t>(tv, 256);   // diagnostics: a consumer thread owns one column of every tile
   int stages = std::max(1, opt.stages);
   const int cps = opt.cps > 0 ? opt.cps : 2;
   const size_t table_bytes = table_smem_bytes(n, p.nnz);
@@ -40,9 +41,8 @@ int launch_tma(const DeviceInfo &dev, StepParams p, const ConstTable *ct, int up
   for (;;) {
     const int parts = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(8, kTmaConsumers / tv)));
     p.uniform_parts = uniform ? parts : 0;
-    p.diag_parts = parts;
     smem = static_cast<size_t>(stages) * arrays * n * tv * 16 + fixed + static_cast<size_t>(p.uniform_parts) * tv * 16;
-    if (p.diag != nullptr) smem += diag_scratch_bytes<float4>(n, static_cast<int>(tv), parts);
+    if (p.diag != nullptr) smem += diag_scratch_bytes<float4>(n, static_cast<int>(tv), has_ring);
     if (smem <= budget) break;
     if (!opt.stages_forced && stages > 2) --stages;
     else if (!opt.tile_cols_forced && tv > 8) tv >>= 1;

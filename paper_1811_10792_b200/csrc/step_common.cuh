@@ -83,7 +83,6 @@ struct StepParams {
   double *diag;
   const float *ring_base;  // slot 0 of the ring (diagnostics read every slot), null when tau == 0
   int tau;
-  int diag_parts;          // interleaved partial sums per column in the diagnostics' column-mean pass
 };
 
 template <int VEC> struct VecT;
@@ -260,83 +259,83 @@ __device__ __forceinline__ CtaTables cta_prologue(const StepParams &p, const Con
   return t;
 }
 
-// ---- fused diagnostics (p.diag != null) ---------------------------------------------------------
-// Shared-memory scratch of the diagnostics, placed by the kernels after their own buffers:
-//   [col_part: 2 * diag_parts * tv vectors][mean_h: tv vectors][mean_x: tv vectors][rowacc: 2n doubles]
+// ---- fused diagnostics (the DIAG instantiations of the step kernels) -----------------------------
+// A thread of either kernel owns the same column c = tid mod tv of every tile (tv <= 256 vectors per row segment
+// is enforced by the launchers when diagnostics are on), and the same set of rows.  So:
+//   * the column sums of the half step (and of the ring) are formed from per-thread partial sums taken while the
+//     half step is computed -- 256 / tv threads share a column; their partials meet in `part` behind the barrier
+//     the kernel has anyway (two buffers by tile parity: no extra barrier);
+//   * the squared deviations of item (row, c) go to a private fp32 slot per item, summed over the tiles without
+//     atomics or shuffles; the slots are reduced per row once, at the end of the kernel.
+// Shared-memory scratch, placed by the kernels after their own buffers:
+//   [part: 2 parities x (1 + HAS_RING) arrays x 256 vectors][slots: n * tv float2 (deviation^2, consensus^2)]
 template <typename V>
 struct DiagScratch {
-  V *col_part;
-  V *mean_h;
-  V *mean_x;
-  double *rowacc;
+  float2 *slots;
+  V *part;
 };
 template <typename V>
-__host__ __device__ inline size_t diag_scratch_bytes(int n, int tv, int parts) {
-  return (static_cast<size_t>(2) * parts * tv + 2 * static_cast<size_t>(tv)) * sizeof(V) + 2 * static_cast<size_t>(n) * sizeof(double) + 16;
+__host__ __device__ inline size_t diag_scratch_bytes(int n, int tv, bool has_ring) {
+  return static_cast<size_t>(n) * tv * sizeof(float2) + static_cast<size_t>(2) * (has_ring ? 2 : 1) * 256 * sizeof(V) + 16;
 }
 template <typename V>
-__device__ __forceinline__ DiagScratch<V> diag_scratch(unsigned char *base, int n, int tv, int parts) {
+__device__ __forceinline__ DiagScratch<V> diag_scratch(unsigned char *base, bool has_ring) {
   DiagScratch<V> s;
-  s.rowacc = reinterpret_cast<double *>((reinterpret_cast<uintptr_t>(base) + 15) & ~uintptr_t{15});
-  s.col_part = reinterpret_cast<V *>(s.rowacc + 2 * n);
-  s.mean_h = s.col_part + static_cast<size_t>(2) * parts * tv;
-  s.mean_x = s.mean_h + tv;
+  s.part = reinterpret_cast<V *>((reinterpret_cast<uintptr_t>(base) + 15) & ~uintptr_t{15});
+  s.slots = reinterpret_cast<float2 *>(s.part + 2 * (has_ring ? 2 : 1) * 256);
   return s;
 }
 
-// Column means of the tile's half step (mean_h) and of everything the nodes hold plus everything in transit
-// (mean_x = mean_h + ring column sums / n; by column-stochasticity this is also the node-wise average AFTER the
-// mix, messages in transit included).  H is the n x tv tile of x^(k+1/2) in shared memory.  `ring_tile` is this
-// step's ring slot in shared memory when the kernel staged it, else null (it is then read from global memory,
-// a read the mix repeats a moment later from L2).  Called by `nthreads` threads with thread index `tid`; the
-// caller synchronises those threads before and after.
-template <int VEC, bool HAS_RING, typename V, typename SyncFn>
-__device__ __forceinline__ void diag_column_means(const StepParams &p, const V *H, const V *ring_tile, int64_t col0,
-                                                  const DiagScratch<V> &ds, int tid, int nthreads, SyncFn sync) {
-  const int n = p.n, tv = 1 << p.log2_tile_vecs, parts = p.diag_parts;
-  const int64_t slot_stride = static_cast<int64_t>(n) * p.ld;
-  for (int idx = tid; idx < tv * parts; idx += nthreads) {
-    const int c = idx & (tv - 1), part = idx >> p.log2_tile_vecs;
-    const int64_t col = col0 + static_cast<int64_t>(c) * VEC;
-    V acc = vzero<V>(), racc = vzero<V>();
-    for (int row = part; row < n; row += parts) acc = vadd(acc, H[(row << p.log2_tile_vecs) + c]);
-    if (HAS_RING && col < p.col_end) {
-      for (int s = 0; s < p.tau; ++s) {
-        const float *slot = p.ring_base + s * slot_stride;
-        const bool staged = ring_tile != nullptr && slot == p.ring_x;
-        for (int row = part; row < n; row += parts)
-          racc = vadd(racc, staged ? ring_tile[(row << p.log2_tile_vecs) + c]
-                                   : ld_inplace(reinterpret_cast<const V *>(slot + static_cast<int64_t>(row) * p.ld + col)));
-      }
-    }
-    ds.col_part[idx] = acc;
-    ds.col_part[parts * tv + idx] = racc;
+// Sum over every ring slot of element (row, col) read from global memory, skipping `skip_slot` (the slot a kernel
+// already holds on chip); slot stride n * ld.
+template <typename V>
+__device__ __forceinline__ V diag_ring_sum(const StepParams &p, int64_t offset, const float *skip_slot) {
+  V acc = vzero<V>();
+  const int64_t slot_stride = static_cast<int64_t>(p.n) * p.ld;
+  for (int s = 0; s < p.tau; ++s) {
+    const float *slot = p.ring_base + s * slot_stride;
+    if (slot != skip_slot) acc = vadd(acc, ld_inplace(reinterpret_cast<const V *>(slot + offset)));
   }
-  sync();
-  const float inv_n = 1.0f / static_cast<float>(n);
-  for (int c = tid; c < tv; c += nthreads) {
-    V acc = ds.col_part[c], racc = ds.col_part[parts * tv + c];
-    for (int part = 1; part < parts; ++part) {
-      acc = vadd(acc, ds.col_part[part * tv + c]);
-      racc = vadd(racc, ds.col_part[(parts + part) * tv + c]);
-    }
-    ds.mean_h[c] = vmul(inv_n, acc);
-    ds.mean_x[c] = vmul(inv_n, vadd(acc, racc));
-  }
-  sync();
+  return acc;
 }
 
-// Adds one item's squared deviations to the per-row accumulators.  Called by ALL lanes of a warp with the same
-// trip count (inactive lanes pass zeros): the `width` = min(32, tv) consecutive lanes that share a row reduce
-// with shuffles, one shared-memory atomic per group.
-__device__ __forceinline__ void diag_accumulate(float dq, float cq, int row, int n, int width, double *rowacc, bool leader_valid) {
-  for (int o = width >> 1; o > 0; o >>= 1) {
-    dq += __shfl_xor_sync(0xffffffffu, dq, o);
-    cq += __shfl_xor_sync(0xffffffffu, cq, o);
+// Column means for this thread's column from the partial sums of the 256 / tv threads that share it:
+// mean_h = (1/n) sum_i h_i, mean_x = mean_h + (1/n) (ring column sum) -- by column-stochasticity the node-wise
+// average AFTER the mix, messages in transit included.
+template <bool HAS_RING, typename V>
+__device__ __forceinline__ void diag_means(const StepParams &p, const V *part_h, const V *part_r, int tid, V *mean_h, V *mean_x) {
+  const int tv = 1 << p.log2_tile_vecs;
+  const int c = tid & (tv - 1);
+  V acc = vzero<V>(), racc = vzero<V>();
+  for (int g = c; g < 256; g += tv) {
+    acc = vadd(acc, part_h[g]);
+    if (HAS_RING) racc = vadd(racc, part_r[g]);
   }
-  if (leader_valid && ((threadIdx.x & 31) & (width - 1)) == 0) {
-    atomicAdd(rowacc + row, static_cast<double>(dq));
-    atomicAdd(rowacc + n + row, static_cast<double>(cq));
+  const float inv_n = 1.0f / static_cast<float>(p.n);
+  *mean_h = vmul(inv_n, acc);
+  *mean_x = vmul(inv_n, vadd(acc, racc));
+}
+
+// End of the kernel: every warp reduces whole rows of the slots and adds them to the global accumulators
+// (fp64 atomics, 2n per CTA).  `nthreads` threads with index `tid` take part.
+__device__ __forceinline__ void diag_flush(const StepParams &p, const float2 *slots, int tid, int nthreads) {
+  const int tv = 1 << p.log2_tile_vecs;
+  const int warp = tid >> 5, lane = tid & 31, nwarps = nthreads >> 5;
+  for (int row = warp; row < p.n; row += nwarps) {
+    float dq = 0.f, cq = 0.f;
+    for (int c = lane; c < tv; c += 32) {
+      const float2 v = slots[row * tv + c];
+      dq += v.x;
+      cq += v.y;
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+      dq += __shfl_xor_sync(0xffffffffu, dq, o);
+      cq += __shfl_xor_sync(0xffffffffu, cq, o);
+    }
+    if (lane == 0) {
+      atomicAdd(p.diag + row, static_cast<double>(dq));
+      atomicAdd(p.diag + p.n + row, static_cast<double>(cq));
+    }
   }
 }
 

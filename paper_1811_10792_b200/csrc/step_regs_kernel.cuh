@@ -14,6 +14,7 @@ sgp_step_regs_kernel(const __grid_constant__ StepParams p, const __grid_constant
   constexpr bool HAS_M = UpdTraits<UPD>::kHasM;
   constexpr bool HAS_V = UpdTraits<UPD>::kHasV;
   constexpr int kItemsPerThread = UpdTraits<UPD>::kItems;
+  constexpr int kDiagArrays = HAS_RING ? 2 : 1;
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int n = p.n;
   const int tv = 1 << p.log2_tile_vecs;
@@ -23,17 +24,15 @@ sgp_step_regs_kernel(const __grid_constant__ StepParams p, const __grid_constant
   V *partial = H0 + (p.single_buffer ? 1 : 2) * tile_items;          // uniform_parts x tv vectors (uniform rows only)
   float *scratch = reinterpret_cast<float *>(partial + p.uniform_parts * tv);
   const CtaTables tab = cta_prologue<HAS_RING>(p, ct, scratch, kThreads);
-  constexpr bool diag = DIAG;      // fused diagnostics: a separate instantiation, so the plain step pays nothing
-  // The diagnostics' scratch sits after the weights and, when it was copied, the table.  Its pointers are
-  // re-derived where they are used (diagnostics only) instead of being kept live through the hot loop.
-  auto diag_ds = [&]() {
-    unsigned char *after = smem_raw + (static_cast<size_t>(p.single_buffer ? 1 : 2) * tile_items + static_cast<size_t>(p.uniform_parts) * tv) * sizeof(V) +
-                           3 * static_cast<size_t>(n) * 4 + (p.table_mode < 2 ? (static_cast<size_t>(n) + 1 + 2 * static_cast<size_t>(p.nnz)) * 4 : 0);
-    return diag_scratch<V>(after, n, tv, p.diag_parts);
-  };
-  if (diag) {
-    const DiagScratch<V> ds = diag_ds();
-    for (int i = threadIdx.x; i < 2 * n; i += kThreads) ds.rowacc[i] = 0.0;
+  // Fused diagnostics (a separate instantiation, so the plain step pays nothing): scratch after the weights
+  // and, when it was copied, the table.
+  DiagScratch<V> ds{};
+  int dbuf = 0;
+  if (DIAG) {
+    unsigned char *after = reinterpret_cast<unsigned char *>(scratch + 3 * n) +
+                           (p.table_mode < 2 ? (static_cast<size_t>(n) + 1 + 2 * static_cast<size_t>(p.nnz)) * 4 : 0);
+    ds = diag_scratch<V>(after, HAS_RING);
+    for (int i = threadIdx.x; i < tile_items; i += kThreads) ds.slots[i] = make_float2(0.f, 0.f);
     __syncthreads();
   }
 
@@ -51,9 +50,11 @@ sgp_step_regs_kernel(const __grid_constant__ StepParams p, const __grid_constant
   for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
     const int64_t col0 = p.col_begin + tile * tile_cols;
     V *H = buf ? H1 : H0;
+    V csum = vzero<V>(), rsum = vzero<V>();      // diagnostics: this thread's share of its column's sums
     // ---- phase 1: local update, all batches of this tile
     for (int base = 0; base < tile_items; base += batch_items) {
       V x[kItemsPerThread], g[kItemsPerThread], u[kItemsPerThread], vv[kItemsPerThread];
+      V rr[DIAG && HAS_RING ? kItemsPerThread : 1];   // diagnostics: everything in transit at this item
       bool ok[kItemsPerThread];
       int64_t off[kItemsPerThread];
 #pragma unroll
@@ -73,6 +74,8 @@ sgp_step_regs_kernel(const __grid_constant__ StepParams p, const __grid_constant
           g[q] = ld_stream(reinterpret_cast<const V *>(p.G + off[q]));
           if (HAS_M) u[q] = ld_inplace(reinterpret_cast<const V *>(p.M + off[q]));
           if (HAS_V) vv[q] = ld_inplace(reinterpret_cast<const V *>(p.V + off[q]));
+          // issued with the batch's other loads (the mix re-reads this step's slot a moment later, from L2)
+          if (DIAG && HAS_RING) rr[q] = diag_ring_sum<V>(p, off[q], nullptr);
         }
       }
 #pragma unroll
@@ -83,15 +86,26 @@ sgp_step_regs_kernel(const __grid_constant__ StepParams p, const __grid_constant
           if (HAS_M) st_stream(reinterpret_cast<V *>(p.M + off[q]), u[q]);
           if (HAS_V) st_stream(reinterpret_cast<V *>(p.V + off[q]), vv[q]);
           H[item] = h;
+          if (DIAG) {
+            csum = vadd(csum, h);
+            if (HAS_RING) rsum = vadd(rsum, rr[q]);
+          }
         } else if (q < q_max && item < tile_items) {
           H[item] = vzero<V>();
         }
       }
     }
+    if (DIAG) {
+      ds.part[(dbuf * kDiagArrays + 0) * 256 + threadIdx.x] = csum;
+      if (HAS_RING) ds.part[(dbuf * kDiagArrays + 1) * 256 + threadIdx.x] = rsum;
+    }
     __syncthreads();
-    if (diag)
-      diag_column_means<VEC, HAS_RING, V>(p, H, static_cast<const V *>(nullptr), col0, diag_ds(), threadIdx.x, kThreads,
-                                          [] { __syncthreads(); });
+    V mean_h = vzero<V>(), mean_x = vzero<V>();
+    if (DIAG) {
+      diag_means<HAS_RING, V>(p, ds.part + (dbuf * kDiagArrays + 0) * 256, ds.part + (dbuf * kDiagArrays + 1) * 256,
+                              threadIdx.x, &mean_h, &mean_x);
+      dbuf ^= 1;
+    }
     // ---- phase 2, all receivers alike (complete graph): one weighted column sum, shared by every row
     if (!HAS_RING && p.uniform_parts > 0) {
       const int parts = p.uniform_parts;
@@ -106,29 +120,27 @@ sgp_step_regs_kernel(const __grid_constant__ StepParams p, const __grid_constant
         partial[idx] = acc;
       }
       __syncthreads();
-      for (int it0 = 0; it0 < tile_items; it0 += kThreads) {
-        const int item = it0 + threadIdx.x;
+      for (int item = threadIdx.x; item < tile_items; item += kThreads) {
         const int row = item >> p.log2_tile_vecs;
         const int c = item & (tv - 1);
         const int64_t col = col0 + static_cast<int64_t>(c) * VEC;
-        float dq = 0.f, cq = 0.f;
-        if (item < tile_items && col < p.col_end) {
+        if (col < p.col_end) {
           const int64_t o = static_cast<int64_t>(row) * ld + col;
           V acc = partial[c];
           for (int part = 1; part < parts; ++part) acc = vadd(acc, partial[part * tv + c]);
           const V z = vmul(tab.inv_w[row], acc);
           st_stream(reinterpret_cast<V *>(p.X + o), acc);
           if (HAS_Z) st_stream(reinterpret_cast<V *>(p.Z + o), z);
-          if (diag) {
-            const DiagScratch<V> ds = diag_ds();
-            dq = vsq(vsub(H[item], ds.mean_h[c]));
-            cq = vsq(vsub(z, ds.mean_x[c]));
+          if (DIAG) {
+            float2 s = ds.slots[item];
+            s.x += vsq(vsub(H[item], mean_h));
+            s.y += vsq(vsub(z, mean_x));
+            ds.slots[item] = s;
           }
         }
-        if (diag) diag_accumulate(dq, cq, row, n, tv < 32 ? tv : 32, diag_ds().rowacc, item < tile_items);
       }
       buf ^= 1;
-      if (p.single_buffer || diag) __syncthreads();
+      if (p.single_buffer) __syncthreads();
       continue;
     }
     // ---- phase 2: gather-mix over the step's in-neighbour lists, ring exchange, de-bias
@@ -151,7 +163,6 @@ sgp_step_regs_kernel(const __grid_constant__ StepParams p, const __grid_constant
         const int row = item >> p.log2_tile_vecs;
         const int c = item & (tv - 1);
         const int64_t col = col0 + static_cast<int64_t>(c) * VEC;
-        float dq = 0.f, cq = 0.f;
         if (q < q_max && item < tile_items && col < p.col_end) {
           const int64_t o = static_cast<int64_t>(row) * ld + col;
           V acc = vzero<V>(), offd = vzero<V>();
@@ -171,23 +182,21 @@ sgp_step_regs_kernel(const __grid_constant__ StepParams p, const __grid_constant
           const V z = vmul(tab.inv_w[row], acc);
           st_stream(reinterpret_cast<V *>(p.X + o), acc);
           if (HAS_Z) st_stream(reinterpret_cast<V *>(p.Z + o), z);
-          if (diag) {
-            const DiagScratch<V> ds = diag_ds();
-            dq = vsq(vsub(H[item], ds.mean_h[c]));
-            cq = vsq(vsub(z, ds.mean_x[c]));
+          if (DIAG) {
+            float2 s = ds.slots[item];
+            s.x += vsq(vsub(H[item], mean_h));
+            s.y += vsq(vsub(z, mean_x));
+            ds.slots[item] = s;
           }
         }
-        if (diag && q < q_max) diag_accumulate(dq, cq, row, n, tv < 32 ? tv : 32, diag_ds().rowacc, item < tile_items);
       }
     }
     buf ^= 1;
-    if (p.single_buffer || diag) __syncthreads();   // the only tile (or the column means) is about to be overwritten
+    if (p.single_buffer) __syncthreads();   // the only tile is about to be overwritten
   }
-  if (diag) {
+  if (DIAG) {
     __syncthreads();
-    const DiagScratch<V> ds = diag_ds();
-    for (int i = threadIdx.x; i < 2 * n; i += kThreads)
-      if (ds.rowacc[i] != 0.0) atomicAdd(p.diag + i, ds.rowacc[i]);
+    diag_flush(p, ds.slots, threadIdx.x, kThreads);
   }
 }
 

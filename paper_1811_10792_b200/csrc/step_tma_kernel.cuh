@@ -123,15 +123,15 @@ sgp_step_tma_kernel(const __grid_constant__ StepParams p, const __grid_constant_
   __shared__ int s_abort;
 
   const CtaTables tab = cta_prologue<HAS_RING>(p, ct, scratch, kTmaThreads);
-  constexpr bool diag = DIAG;      // fused diagnostics: a separate instantiation
+  // Fused diagnostics (a separate instantiation): scratch after the weights and, when it was copied, the table.
+  constexpr int kDiagArrays = HAS_RING ? 2 : 1;
   DiagScratch<float4> ds{};
-  if (diag) {
+  if (DIAG) {
     unsigned char *after = reinterpret_cast<unsigned char *>(scratch + 3 * n) +
                            (p.table_mode < 2 ? (static_cast<size_t>(n) + 1 + 2 * static_cast<size_t>(p.nnz)) * 4 : 0);
-    ds = diag_scratch<float4>(after, n, tv, p.diag_parts);
-    for (int i = threadIdx.x; i < 2 * n; i += kTmaThreads) ds.rowacc[i] = 0.0;
+    ds = diag_scratch<float4>(after, HAS_RING);
+    for (int i = threadIdx.x; i < tile_items; i += kTmaThreads) ds.slots[i] = make_float2(0.f, 0.f);
   }
-  const int diag_width = tv < 32 ? tv : 32;
   if (threadIdx.x == 0) {
     for (int s = 0; s < stages; ++s) {
       mbar_init(full_bar + s, 1);
@@ -230,6 +230,7 @@ sgp_step_tma_kernel(const __grid_constant__ StepParams p, const __grid_constant_
       const float4 *Vs = Xs + static_cast<size_t>(kIdxV) * tile_items;
       const float4 *Rs = Xs + static_cast<size_t>(kIdxR) * tile_items;
       // phase 1: local update; x^(k+1/2) replaces x in the stage
+      float4 csum = make_float4(0.f, 0.f, 0.f, 0.f), rsum = csum;   // diagnostics: this thread's share of its column's sums
       for (int item = ctid; item < tile_items; item += kTmaConsumers) {
         const int row = item >> p.log2_tile_vecs;
         const int c = item & (tv - 1);
@@ -241,12 +242,23 @@ sgp_step_tma_kernel(const __grid_constant__ StepParams p, const __grid_constant_
           if (HAS_M) st_stream(reinterpret_cast<float4 *>(p.M + static_cast<int64_t>(row) * ld + col), u);
           if (HAS_V) st_stream(reinterpret_cast<float4 *>(p.V + static_cast<int64_t>(row) * ld + col), v2);
           Xs[item] = h;
+          if (DIAG) {
+            csum = vadd(csum, h);
+            // everything in transit in this column: this step's slot is in the stage, the others come from HBM
+            if (HAS_RING) rsum = vadd(rsum, vadd(Rs[item], diag_ring_sum<float4>(p, static_cast<int64_t>(row) * ld + col, p.ring_x)));
+          }
         }
       }
+      const int dbuf = static_cast<int>(it & 1);
+      if (DIAG) {
+        ds.part[(dbuf * kDiagArrays + 0) * 256 + ctid] = csum;
+        if (HAS_RING) ds.part[(dbuf * kDiagArrays + 1) * 256 + ctid] = rsum;
+      }
       consumer_barrier();
-      if (diag)
-        diag_column_means<4, HAS_RING, float4>(p, Xs, HAS_RING ? Rs : static_cast<const float4 *>(nullptr), col0, ds, ctid,
-                                               kTmaConsumers, [] { consumer_barrier(); });
+      float4 mean_h = make_float4(0.f, 0.f, 0.f, 0.f), mean_x = mean_h;
+      if (DIAG)
+        diag_means<HAS_RING, float4>(p, ds.part + (dbuf * kDiagArrays + 0) * 256, ds.part + (dbuf * kDiagArrays + 1) * 256, ctid,
+                                     &mean_h, &mean_x);
       if (!HAS_RING && p.uniform_parts > 0) {
         // all receivers alike (complete graph): one weighted column sum, shared by every row
         const int parts = p.uniform_parts;
@@ -258,25 +270,24 @@ sgp_step_tma_kernel(const __grid_constant__ StepParams p, const __grid_constant_
           partial[idx] = acc;
         }
         consumer_barrier();
-        for (int it0 = 0; it0 < tile_items; it0 += kTmaConsumers) {
-          const int item = it0 + ctid;
+        for (int item = ctid; item < tile_items; item += kTmaConsumers) {
           const int row = item >> p.log2_tile_vecs;
           const int c = item & (tv - 1);
           const int64_t col = col0 + static_cast<int64_t>(c) * 4;
-          float dq = 0.f, cq = 0.f;
-          if (item < tile_items && col < p.col_end) {
+          if (col < p.col_end) {
             const int64_t o = static_cast<int64_t>(row) * ld + col;
             float4 acc = partial[c];
             for (int part = 1; part < parts; ++part) acc = vadd(acc, partial[part * tv + c]);
             const float4 z = vmul(tab.inv_w[row], acc);
             st_stream(reinterpret_cast<float4 *>(p.X + o), acc);
             if (HAS_Z) st_stream(reinterpret_cast<float4 *>(p.Z + o), z);
-            if (diag) {
-              dq = vsq(vsub(Xs[item], ds.mean_h[c]));
-              cq = vsq(vsub(z, ds.mean_x[c]));
+            if (DIAG) {
+              float2 sq = ds.slots[item];
+              sq.x += vsq(vsub(Xs[item], mean_h));
+              sq.y += vsq(vsub(z, mean_x));
+              ds.slots[item] = sq;
             }
           }
-          if (diag) diag_accumulate(dq, cq, row, n, diag_width, ds.rowacc, item < tile_items);
         }
         consumer_barrier();          // the partial sums are rewritten by the next tile
         fence_proxy_async_smem();
@@ -285,13 +296,11 @@ sgp_step_tma_kernel(const __grid_constant__ StepParams p, const __grid_constant_
         continue;
       }
       // phase 2: gather-mix, ring exchange, de-bias
-      for (int it0 = 0; it0 < tile_items; it0 += kTmaConsumers) {
-        const int item = it0 + ctid;
+      for (int item = ctid; item < tile_items; item += kTmaConsumers) {
         const int row = item >> p.log2_tile_vecs;
         const int c = item & (tv - 1);
         const int64_t col = col0 + static_cast<int64_t>(c) * 4;
-        float dq = 0.f, cq = 0.f;
-        if (item < tile_items && col < p.col_end) {
+        if (col < p.col_end) {
           const int64_t o = static_cast<int64_t>(row) * ld + col;
           float4 acc = make_float4(0.f, 0.f, 0.f, 0.f), offd = acc;
           const int e1 = tab.rowptr[row + 1];
@@ -310,23 +319,22 @@ sgp_step_tma_kernel(const __grid_constant__ StepParams p, const __grid_constant_
           const float4 z = vmul(tab.inv_w[row], acc);
           st_stream(reinterpret_cast<float4 *>(p.X + o), acc);
           if (HAS_Z) st_stream(reinterpret_cast<float4 *>(p.Z + o), z);
-          if (diag) {
-            dq = vsq(vsub(Xs[item], ds.mean_h[c]));
-            cq = vsq(vsub(z, ds.mean_x[c]));
+          if (DIAG) {
+            float2 sq = ds.slots[item];
+            sq.x += vsq(vsub(Xs[item], mean_h));
+            sq.y += vsq(vsub(z, mean_x));
+            ds.slots[item] = sq;
           }
         }
-        if (diag) diag_accumulate(dq, cq, row, n, diag_width, ds.rowacc, item < tile_items);
       }
-      if (diag) consumer_barrier();   // the column means are rewritten by the next tile
       // the stage may be refilled by the async proxy once every consumer warp has released it
       fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(empty_bar + s);
     }
-    if (diag) {
+    if (DIAG) {
       consumer_barrier();            // every consumer is here: all leave the loop together, also on an aborted run
-      for (int i = ctid; i < 2 * n; i += kTmaConsumers)
-        if (ds.rowacc[i] != 0.0) atomicAdd(p.diag + i, ds.rowacc[i]);
+      diag_flush(p, ds.slots, ctid, kTmaConsumers);
     }
   }
 }

@@ -1,0 +1,225 @@
+"""One node per GPU, exercised on ONE device: every rank has its own message slots and rows (separate allocations),
+the mix kernels read their in-neighbours' slots through pointer tables exactly as they would through NVLink peer
+mappings.  Parity: element by element against the float64 oracle, and bit for bit against the stacked
+all-nodes-on-one-GPU step (same CSR order, same FMA chain).  App. C; Alg. 1 lines 4-8; Alg. 2."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from gpu_runner import DEV
+from parity_util import assert_close, graph_desc, oracle_P_of_k
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_1811_10792_b200 import build
+    build.build()
+    from paper_1811_10792_b200 import binding as b
+    return b
+
+
+@pytest.fixture(scope="module")
+def inputs():
+    from paper_1811_10792_b200 import inputs as i
+    return i
+
+
+def _run_both(binding, inputs, w, K, offset=0, write_z=True, flags=0):
+    """K steps in loopback one-node-per-GPU mode and K steps of the stacked step on the same inputs."""
+    from paper_1811_10792_b200 import rowshard
+    n, d = w.n, w.d
+    X = inputs.initial_x(w, device=DEV).contiguous()
+    x0 = X.cpu().numpy().astype(np.float64)
+    W = torch.ones(n, device=DEV)
+    M = torch.zeros_like(X)
+    Z = torch.full_like(X, float("nan"))
+    G = torch.empty_like(X)
+
+    def row(fill):                       # separate allocations per rank, optionally misaligned (scalar path)
+        buf = torch.full((d + offset + 8,), fill, device=DEV)
+        return buf, buf[offset:offset + d]
+    xs, ms, zs, gs = ([row(float("nan")) for _ in range(n)] for _ in range(4))
+    ws = [torch.ones(1, device=DEV) for _ in range(n)]
+    for r in range(n):
+        xs[r][1].copy_(X[r])
+        ms[r][1].zero_()
+    grads = []
+    with binding.Sgp(n, d, graph_desc(w, binding), tau=w.tau, flags=flags) as h, \
+            rowshard.LoopbackGroup(n, d, graph_desc(w, binding), tau=w.tau, flags=flags) as grp:
+        for k in range(K):
+            inputs.gradient(w, k, G)
+            grads.append(G.cpu().numpy().astype(np.float64))
+            for r in range(n):
+                gs[r][1].copy_(G[r])
+            grp.step([t[1] for t in xs], ws, [t[1] for t in ms], [t[1] for t in gs],
+                     [t[1] for t in zs] if write_z else None, k, w.lr, w.momentum, w.weight_decay, w.nesterov)
+            h.step(X, W, M if w.momentum else None, G, Z if write_z else None, k, w.lr, w.momentum, w.weight_decay,
+                   w.nesterov)
+        torch.cuda.synchronize()
+        assert grp.device_status() == 0 and h.device_status() == 0
+    for name, bufs in (("x", xs), ("m", ms), ("z", zs)):               # nothing outside the rows was touched
+        for buf, view in bufs:
+            full = buf.cpu().numpy()
+            assert np.all(np.isnan(full[:offset])) and np.all(np.isnan(full[offset + d:])), name
+    got = dict(X=torch.stack([t[1] for t in xs]), M=torch.stack([t[1] for t in ms]), Z=torch.stack([t[1] for t in zs]),
+               W=torch.cat(ws))
+    return x0, grads, got, dict(X=X, M=M, Z=Z, W=W)
+
+
+CASES = [
+    dict(n=8, d=4_100, graph="exp", peers=1, tau=0, momentum=0.9),
+    dict(n=8, d=4_100, graph="exp", peers=2, tau=0, momentum=0.0),
+    dict(n=8, d=4_101, graph="exp", peers=1, tau=1, momentum=0.9),              # ragged end of the row
+    dict(n=16, d=9_000, graph="random", tau=0, momentum=0.9),                   # irregular in-degree, w != 1
+    dict(n=16, d=9_000, graph="random", tau=2, momentum=0.9),
+    dict(n=32, d=2_051, graph="random", tau=3, momentum=0.9, nesterov=False),
+    dict(n=4, d=1_000, graph="bipartite", tau=0, momentum=0.9),
+    dict(n=2, d=515, graph="exp", peers=1, tau=1, momentum=0.0),
+    dict(n=1, d=300, graph="exp", peers=1, tau=0, momentum=0.9),
+    dict(n=5, d=1_003, graph="random", tau=1, momentum=0.9, offset=1),          # misaligned rows: scalar kernels
+    dict(n=5, d=1_003, graph="random", tau=0, momentum=0.9, offset=3),
+]
+
+
+@pytest.mark.parametrize("case", CASES)
+def test_loopback_ranks_match_oracle_and_stacked_step(binding, inputs, case):
+    from oracle import sgp as osgp
+    base = inputs.sweep_workload(case["n"], case["d"])
+    w = dataclasses.replace(base, graph=case["graph"], peers=case.get("peers", 1), tau=case["tau"],
+                            momentum=case["momentum"], nesterov=case.get("nesterov", True), weight_decay=1e-3)
+    K = 7
+    x0, grads, got, stacked = _run_both(binding, inputs, w, K, offset=case.get("offset", 0))
+    st = osgp.sgp_run(x0, K, oracle_P_of_k(w), lambda k, z: grads[k], w.lr, momentum=w.momentum, nesterov=w.nesterov,
+                      weight_decay=w.weight_decay, tau=w.tau)
+    assert_close("X", got["X"].cpu().numpy(), st.x)
+    assert_close("Z", got["Z"].cpu().numpy(), st.z)
+    assert_close("W", got["W"].cpu().numpy(), st.w)
+    if w.momentum:
+        assert_close("M", got["M"].cpu().numpy(), st.u)
+    for name in ("X", "Z", "W") + (("M",) if w.momentum else ()):
+        assert torch.equal(got[name], stacked[name]), f"{name}: one-node-per-GPU and stacked results differ"
+    if case["graph"] == "random":
+        assert np.ptp(got["W"].cpu().numpy()) > 1e-3                    # the weight path is exercised
+
+
+def test_loopback_without_z_and_biased(binding, inputs):
+    w = dataclasses.replace(inputs.sweep_workload(8, 2_000), tau=1)
+    x0, grads, got, stacked = _run_both(binding, inputs, w, 5, write_z=False)
+    assert torch.isnan(got["Z"]).all().item() and torch.equal(got["X"], stacked["X"])
+    x0, grads, got, stacked = _run_both(binding, inputs, w, 5, flags=binding.SGP_FLAG_BIASED)
+    assert torch.equal(got["Z"], got["X"]) and torch.equal(got["X"], stacked["X"])
+
+
+def test_rank_argument_checks(binding, inputs):
+    g = binding.GraphDesc.exp_peers(1)
+    for bad in (dict(rank=4, world=4), dict(rank=-1, world=4), dict(rank=0, world=0), dict(rank=0, world=257)):
+        with pytest.raises(binding.SgpError) as e:
+            binding.SgpRank(bad["rank"], bad["world"], 100, g)
+        assert e.value.code == binding.SGP_ERR_ARG
+    x = torch.zeros(100, device=DEV); w = torch.ones(1, device=DEV); gr = torch.zeros(100, device=DEV)
+    r0 = binding.SgpRank(0, 4, 100, g, tau=0)
+    r1 = binding.SgpRank(1, 4, 100, g, tau=1)
+    try:
+        with pytest.raises(binding.SgpError) as e:
+            r0.step_overlap(x, w, None, gr, None, 0, 0.1)               # tau = 0: the peers' messages are not there yet
+        assert e.value.code == binding.SGP_ERR_STATE
+        with pytest.raises(binding.SgpError) as e:
+            r1.mix(x, w, None, 0)
+        assert e.value.code == binding.SGP_ERR_STATE
+        r0.update(x, w, None, gr, 0, 0.1)
+        with pytest.raises(binding.SgpError) as e:                     # in-neighbour 3 was never mapped
+            r0.mix(x, w, None, 0)
+        assert e.value.code == binding.SGP_ERR_STATE
+        with pytest.raises(binding.SgpError) as e:
+            r0.update(x, w, None, gr, 0, 0.1, momentum=0.9)             # momentum without m
+        assert e.value.code == binding.SGP_ERR_ARG
+        torch.cuda.synchronize()
+    finally:
+        r0.close(); r1.close()
+    # complete graph on 64 nodes: in-degree above what one mix takes
+    sched = binding.Schedule(64, binding.GraphDesc.complete())
+    with pytest.raises(binding.SgpError) as e:
+        binding.rank_plan(sched, 0, 0, 0)
+    assert e.value.code == binding.SGP_ERR_ARG
+
+
+def test_ipc_export_of_the_message_block(binding):
+    """Exporting a rank's slots gives a 64-byte handle; opening one's own handle inside the exporting process is
+    the runtime's call to refuse or allow: either way it comes back as a code, not a crash."""
+    g = binding.GraphDesc.exp_peers(1)
+    r0 = binding.SgpRank(0, 2, 1 << 16, g)
+    try:
+        ptr, size = r0.message_block()
+        assert size >= 2 * 4 * (1 << 16)
+        handle = binding.ipc_export(ptr)
+        assert len(handle) == binding.SGP_IPC_HANDLE_BYTES and any(handle)
+        try:
+            mapped = binding.ipc_open(handle)
+        except binding.SgpError as e:
+            assert e.code == binding.SGP_ERR_CUDA
+        else:
+            binding.ipc_close(mapped)
+        torch.cuda.synchronize()
+    finally:
+        r0.close()
+
+
+# ---------------------------------------------------------------- two processes, CUDA IPC, one device
+def _ipc_worker(rank, world, port, tau, d, K, out):
+    """One process per rank, both on device 0: the peers' message slots are reached through CUDA IPC mappings, the
+    per-step barrier is a host barrier (gloo).  No kernel waits on another process's kernel."""
+    import os
+    import sys
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    from conftest import ROOT
+    sys.path.insert(0, ROOT)
+    import torch.distributed as dist
+    from paper_1811_10792_b200 import binding as b, inputs as inp, rowshard
+    torch.cuda.set_device(0)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        w = dataclasses.replace(inp.sweep_workload(world, d), graph="exp", peers=1, tau=tau)
+        X = inp.initial_x(w, device=DEV).contiguous()
+        G = torch.empty_like(X)
+        x, m, z = X[rank].clone(), torch.zeros(d, device=DEV), torch.empty(d, device=DEV)
+        wt = torch.ones(1, device=DEV)
+        node = rowshard.DistributedRank(d, b.GraphDesc.exp_peers(1), tau=tau)
+        for k in range(K):
+            inp.gradient(w, k, G)
+            node.step(x, wt, m, G[rank].clone(), z, k, w.lr, w.momentum, w.weight_decay, True)
+        torch.cuda.synchronize()
+        dist.barrier()
+        out[rank] = (x.cpu().numpy(), z.cpu().numpy(), m.cpu().numpy(), float(wt.item()), node.node.device_status())
+        dist.barrier()
+        node.close()
+    finally:
+        dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("tau", [0, 1])
+def test_two_processes_share_slots_through_cuda_ipc(binding, inputs, tau):
+    import torch.multiprocessing as mp
+    from oracle import sgp as osgp
+    world, d, K = 2, 6_004, 5
+    ctx = mp.get_context("spawn")
+    with ctx.Manager() as mgr:
+        out = mgr.dict()
+        mp.spawn(_ipc_worker, args=(world, 29950 + tau, tau, d, K, out), nprocs=world, join=True)
+        res = dict(out)
+    w = dataclasses.replace(inputs.sweep_workload(world, d), graph="exp", peers=1, tau=tau)
+    x0 = inputs.initial_x(w, device=DEV).cpu().numpy().astype(np.float64)
+    G = torch.empty((world, d), device=DEV)
+    grads = [inputs.gradient(w, k, G).cpu().numpy().astype(np.float64) for k in range(K)]
+    st = osgp.sgp_run(x0, K, oracle_P_of_k(w), lambda k, z: grads[k], w.lr, momentum=w.momentum, nesterov=True,
+                      weight_decay=w.weight_decay, tau=tau)
+    for r in range(world):
+        x, z, m, wt, status = res[r]
+        assert status == 0
+        assert_close(f"x[{r}]", x, st.x[r])
+        assert_close(f"z[{r}]", z, st.z[r])
+        assert_close(f"m[{r}]", m, st.u[r])
+        assert abs(wt - st.w[r]) <= 1e-6
