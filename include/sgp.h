@@ -198,6 +198,12 @@ int sgp_step_host(sgp_handle *h, float *d_X, float *d_W, float *d_M, const float
                   float *d_G, float *d_Z, int64_t k, float lr, float momentum, float weight_decay,
                   int nesterov, int64_t chunk_cols, void *stream);
 
+/* sgp_step_adam_host: the Adam iteration of sgp_step_adam with gradients and de-biased parameters in HOST memory,
+ * pipelined like sgp_step_host (Sec. 6.2 / App. C.1 optimiser; same chunking, streams and synchronisation). */
+int sgp_step_adam_host(sgp_handle *h, float *d_X, float *d_W, float *d_M1, float *d_M2, const float *h_G, float *h_Z,
+                       float *d_G, float *d_Z, int64_t k, int64_t t, float lr, float beta1, float beta2, float eps,
+                       float weight_decay, int64_t chunk_cols, void *stream);
+
 /* Zeroes the delay ring (messages in transit are dropped: use only to restart a run). */
 int sgp_reset(sgp_handle *h, void *stream);
 /* Checkpointing of the in-transit messages: d_ring_x is tau*n*ld floats, d_ring_w is tau*n floats
@@ -261,7 +267,10 @@ int sgp_param_deviation(sgp_handle *h, const float *d_A, double *h_dev, void *st
 /*
  * Tuning knobs for experiments (defaults are chosen per problem shape):
  *   "variant"      0 = automatic, 1 = register-staged kernel, 2 = TMA pipelined kernel fed by 2-D tensor
- *                  maps, 3 = the same kernel fed by one bulk copy per row segment (no tensor maps)
+ *                  maps, 3 = the same kernel fed by one bulk copy per row segment (no tensor maps), 4 = the
+ *                  thread-block-cluster kernel (a cluster of CTAs shares a tile through distributed shared memory)
+ *                  -- measured slower than variant 1 at every shape tried, never chosen automatically
+ *   "cluster"      CTAs per cluster of variant 4: 0 = 2, 1 = do not use clusters, 2 or 4
  *   "tile_cols"    columns per tile (multiple of 4; 0 = automatic)
  *   "ctas_per_sm"  persistent CTAs per SM (0 = automatic)
  *   "stages"       shared-memory stages of the bulk-copy pipeline (0 = automatic, at most 8)

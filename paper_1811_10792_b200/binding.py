@@ -33,7 +33,7 @@ EXPORTS = [
     "sgp_step_adam", "sgp_param_deviation", "sgp_set_graph", "sgp_colsum", "sgp_get_diagnostics",
     "sgp_rank_plan", "sgp_rank_create", "sgp_rank_destroy", "sgp_rank_get_schedule", "sgp_rank_message_block",
     "sgp_rank_set_peers", "sgp_rank_update", "sgp_rank_mix", "sgp_rank_step_overlap", "sgp_rank_device_status",
-    "sgp_ipc_export", "sgp_ipc_open", "sgp_ipc_close",
+    "sgp_ipc_export", "sgp_ipc_open", "sgp_ipc_close", "sgp_step_adam_host",
 ]
 SGP_RANK_MAX_SOURCES = 32
 SGP_IPC_HANDLE_BYTES = 64
@@ -81,6 +81,7 @@ def _load() -> C.CDLL:
         "sgp_debias": [vp, vp, vp, vp, vp],
         "sgp_step_adam": [vp, vp, vp, vp, vp, vp, vp, i64, i64, f32, f32, f32, f32, f32, vp],
         "sgp_step_host": [vp, vp, vp, vp, vp, vp, vp, vp, i64, f32, f32, f32, i32, i64, vp],
+        "sgp_step_adam_host": [vp, vp, vp, vp, vp, vp, vp, vp, vp, i64, i64, f32, f32, f32, f32, f32, i64, vp],
         "sgp_reset": [vp, vp],
         "sgp_ring_export": [vp, vp, vp, vp],
         "sgp_ring_import": [vp, vp, vp, vp],
@@ -311,6 +312,13 @@ class Sgp:
         _check(_lib.sgp_step_host(self._h, _ptr(X), _ptr(W), _ptr(M), _ptr(h_G), _ptr(h_Z), _ptr(d_G), _ptr(d_Z),
                                   k, lr, momentum, weight_decay, int(bool(nesterov)), chunk_cols,
                                   _stream_ptr(stream)), "sgp_step_host")
+
+    def step_adam_host(self, X, W, M1, M2, h_G, h_Z, d_G, d_Z, k: int, t: int, lr: float, beta1: float = 0.9,
+                       beta2: float = 0.999, eps: float = 1e-8, weight_decay: float = 0.0, chunk_cols: int = 0,
+                       stream=None) -> None:
+        _check(_lib.sgp_step_adam_host(self._h, _ptr(X), _ptr(W), _ptr(M1), _ptr(M2), _ptr(h_G), _ptr(h_Z), _ptr(d_G),
+                                       _ptr(d_Z), k, t, lr, beta1, beta2, eps, weight_decay, chunk_cols,
+                                       _stream_ptr(stream)), "sgp_step_adam_host")
 
     def reset(self, stream=None) -> None:
         _check(_lib.sgp_reset(self._h, _stream_ptr(stream)), "sgp_reset")

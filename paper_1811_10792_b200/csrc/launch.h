@@ -77,4 +77,16 @@ using TensorMapFn = bool (*)(void *ctx, const float *base, int box_cols, CUtenso
 int launch_tma(const DeviceInfo &dev, StepParams p, const ConstTable *ct, int upd, bool uniform_rows,
                const TmaOptions &opt, TensorMapFn map_fn, void *map_ctx, cudaStream_t stream, LaunchRecord *rec);
 
+struct ClusterOptions {
+  int cluster_size = 4;           // CTAs per cluster: 2 or 4
+  int64_t tile_cols = 256;
+  bool tile_cols_forced = false;
+  int max_clusters = 0;           // 0 = as many as are resident
+};
+// One launch of the thread-block-cluster kernel (many nodes; 128-bit preconditions, no shared-column-sum path, no
+// diagnostics).  Returns SGP_ERR_STATE when clusters of this shape cannot be resident; the caller then uses the
+// register-staged kernel.
+int launch_cluster(const DeviceInfo &dev, StepParams p, const ConstTable *ct, int upd, const ClusterOptions &opt,
+                   cudaStream_t stream, LaunchRecord *rec);
+
 }  // namespace sgp

@@ -47,7 +47,7 @@ struct sgp_handle {
   double *d_stats = nullptr;    // kDevStatsCount doubles
   double *d_expect = nullptr;   // d doubles, allocated when "check_steps" is switched on
   int64_t opt_variant = 0, opt_tile_cols = 0, opt_ctas_per_sm = 0, opt_stages = 0, opt_l2_hint = 0, opt_single_buffer = 0, opt_wait_limit_ms = 0,
-          opt_inject_stall = 0, opt_send_period = 1, opt_diagnostics = 0, opt_check_steps = 0;
+          opt_inject_stall = 0, opt_send_period = 1, opt_diagnostics = 0, opt_check_steps = 0, opt_cluster = 0;
   sgp::LaunchRecord last;       // of the most recent step launch
   int64_t launches = 0;         // step kernels launched so far
   bool diag_valid = false;      // a step with diagnostics has been enqueued since the last reset
@@ -173,7 +173,7 @@ void fill_params(const sgp_handle *h, const StepArgs &a, int64_t c0, int64_t c1,
 
 // Launch plan of one step: which kernel, how wide a tile, how deep a pipeline, how many CTAs per SM.
 struct Plan {
-  int variant;        // 1 register-staged, 2 TMA with tensor maps, 3 TMA with per-row bulk copies
+  int variant;        // 1 register-staged, 2 TMA with tensor maps, 3 TMA with per-row bulk copies, 4 thread-block cluster
   int64_t tile_cols;  // 0 = kernel default
   int stages;
   int cps;
@@ -214,13 +214,13 @@ Plan make_plan(const sgp_handle *h, int arrays, bool has_m, int nnz, bool vec) {
   }
   if (h->opt_variant > 0 && (h->opt_variant == 1) != (pl.variant == 1)) {
     // the caller forces the other kernel family: take that family's defaults
-    if (h->opt_variant == 1) {
+    if (h->opt_variant == 1 || h->opt_variant == 4) {
       pl = Plan{1, vec ? sgp::regs_tile_cols(h->n, 4 * 1024) : 0, 2, 0};
     } else {
       pl = Plan{static_cast<int>(h->opt_variant), 256, 2, 2};
     }
   }
-  if (h->opt_variant > 0) pl.variant = static_cast<int>(h->opt_variant);
+  if (h->opt_variant > 0 && h->opt_variant < 4) pl.variant = static_cast<int>(h->opt_variant);
   if (h->opt_tile_cols > 0) pl.tile_cols = h->opt_tile_cols;
   if (h->opt_stages > 0) pl.stages = static_cast<int>(h->opt_stages);
   if (h->opt_ctas_per_sm > 0) pl.cps = static_cast<int>(h->opt_ctas_per_sm);
@@ -332,7 +332,28 @@ int launch_step_range(sgp_handle *h, const StepArgs &a, int64_t c0, int64_t c1, 
     // short rows (fewer 1 KB tiles than SMs): the register kernel with narrow tiles spreads them better
     if (h->opt_variant == 0 && pl.variant >= 2 && (vec_end - c0) < int64_t{256} * h->dev.sm_count) pl = Plan{1, 256, 2, 0};
     int rc = SGP_ERR_STATE;
-    if (pl.variant >= 2) rc = launch_tma(h, a, pl, c0, vec_end, update_w && vec_end == c1, stream);
+    // Opt-in (variant 4): a cluster of CTAs shares the tile through distributed shared memory, so that row segments
+    // stay 1 KB long at n = 256 (256 bytes with one CTA).  Measured slower than the one-CTA kernel at every shape
+    // tried (n = 256, d = 1e7: 0.77 of the copy bandwidth with 4 CTAs, 0.86 with 2, against 0.93; n = 64..128:
+    // 0.73-0.87 against 0.92-0.96): two cluster barriers per tile and remote-shared-memory latency in the
+    // gather's dependent chain cost more than the longer segments return.  Never chosen automatically.
+    const size_t slot = slot_of(h, a.k);
+    const bool cluster_ok = !h->opt_diagnostics && !(h->tau == 0 && csr_of(h, slot).uniform_rows) && h->n >= 2;
+    const bool want_cluster = h->opt_variant == 4 && h->opt_cluster != 1;
+    if (cluster_ok && want_cluster) {
+      StepParams p{};
+      fill_params(h, a, c0, vec_end, update_w && vec_end == c1, &p);
+      sgp::ClusterOptions copt;
+      copt.cluster_size = h->opt_cluster >= 2 ? static_cast<int>(h->opt_cluster) : 2;
+      if (h->opt_tile_cols > 0) {
+        copt.tile_cols = h->opt_tile_cols;
+        copt.tile_cols_forced = true;
+      }
+      sgp::LaunchRecord rec;
+      rc = sgp::launch_cluster(h->dev, p, h->const_ok[slot] ? &h->const_tables[slot] : nullptr, a.upd, copt, stream, &rec);
+      record_launch(h, rec, rc);
+    }
+    if (rc == SGP_ERR_STATE && pl.variant >= 2) rc = launch_tma(h, a, pl, c0, vec_end, update_w && vec_end == c1, stream);
     if (rc == SGP_ERR_STATE) {
       Plan fallback = pl;
       if (pl.variant >= 2 && h->opt_ctas_per_sm == 0) fallback.cps = 0;
@@ -489,6 +510,64 @@ int refresh_status(sgp_handle *h, unsigned *out) {
   return SGP_OK;
 }
 
+// The host-buffer step: column chunks pipelined over three streams (H2D of chunk c+1, fused step on chunk c, D2H of
+// chunk c-1); `a` carries the device arrays and the optimiser, a.G / a.Z are the device staging arrays.
+int run_host_step(sgp_handle *h, const StepArgs &a, const float *h_G, float *h_Z, int64_t chunk_cols, void *stream) {
+  float *d_G = const_cast<float *>(a.G);
+  float *d_Z = a.Z;
+  int rc = SGP_OK;
+  if (h->seen_status & kWaitBits) return SGP_ERR_DEVICE;
+  if (h->seen_status & sgp::kStatusZeroWeight) return SGP_ERR_ZERO_WEIGHT;
+  if (h->s_h2d == nullptr) {
+    SGP_CUDA_TRY(h, cudaStreamCreateWithFlags(&h->s_h2d, cudaStreamNonBlocking));
+    SGP_CUDA_TRY(h, cudaStreamCreateWithFlags(&h->s_compute, cudaStreamNonBlocking));
+    SGP_CUDA_TRY(h, cudaStreamCreateWithFlags(&h->s_d2h, cudaStreamNonBlocking));
+    SGP_CUDA_TRY(h, cudaEventCreateWithFlags(&h->ev_entry, cudaEventDisableTiming));
+  }
+  // default chunk: about 64 MB of gradient per chunk, a multiple of 1024 columns
+  if (chunk_cols <= 0) chunk_cols = std::max<int64_t>(1024, (int64_t{64} << 20) / (4 * h->n) / 1024 * 1024);
+  chunk_cols = (chunk_cols + 3) / 4 * 4;
+  const int64_t nchunks = (h->d + chunk_cols - 1) / chunk_cols;
+  while (static_cast<int64_t>(h->ev_in.size()) < nchunks) {
+    cudaEvent_t ev_a = nullptr, ev_b = nullptr;
+    SGP_CUDA_TRY(h, cudaEventCreateWithFlags(&ev_a, cudaEventDisableTiming));
+    h->ev_in.push_back(ev_a);
+    SGP_CUDA_TRY(h, cudaEventCreateWithFlags(&ev_b, cudaEventDisableTiming));
+    h->ev_done.push_back(ev_b);
+  }
+  // what the caller already enqueued on its stream (it may produce X, W, M or read d_G, d_Z) comes first:
+  // an event wait on the device, not a host synchronisation
+  SGP_CUDA_TRY(h, cudaEventRecord(h->ev_entry, static_cast<cudaStream_t>(stream)));
+  SGP_CUDA_TRY(h, cudaStreamWaitEvent(h->s_h2d, h->ev_entry, 0));
+  SGP_CUDA_TRY(h, cudaStreamWaitEvent(h->s_compute, h->ev_entry, 0));
+  SGP_CUDA_TRY(h, cudaStreamWaitEvent(h->s_d2h, h->ev_entry, 0));
+  if (h->opt_diagnostics) {
+    SGP_CUDA_TRY(h, cudaMemsetAsync(h->d_stats + kDevStatsDiag, 0, 2 * static_cast<size_t>(h->n) * sizeof(double), h->s_compute));
+    h->diag_valid = true;
+  }
+  const size_t pitch = static_cast<size_t>(h->ld) * sizeof(float);
+  for (int64_t c = 0; c < nchunks; ++c) {
+    const int64_t c0 = c * chunk_cols, c1 = std::min(h->d, c0 + chunk_cols);
+    const size_t width = static_cast<size_t>(c1 - c0) * sizeof(float);
+    SGP_CUDA_TRY(h, cudaMemcpy2DAsync(d_G + c0, pitch, h_G + c0, pitch, width, static_cast<size_t>(h->n),
+                                      cudaMemcpyHostToDevice, h->s_h2d));
+    SGP_CUDA_TRY(h, cudaEventRecord(h->ev_in[static_cast<size_t>(c)], h->s_h2d));
+    SGP_CUDA_TRY(h, cudaStreamWaitEvent(h->s_compute, h->ev_in[static_cast<size_t>(c)], 0));
+    rc = launch_step_range(h, a, c0, c1, c == nchunks - 1, h->s_compute);
+    if (rc != SGP_OK) return rc;
+    if (h_Z != nullptr) {
+      SGP_CUDA_TRY(h, cudaEventRecord(h->ev_done[static_cast<size_t>(c)], h->s_compute));
+      SGP_CUDA_TRY(h, cudaStreamWaitEvent(h->s_d2h, h->ev_done[static_cast<size_t>(c)], 0));
+      SGP_CUDA_TRY(h, cudaMemcpy2DAsync(h_Z + c0, pitch, d_Z + c0, pitch, width, static_cast<size_t>(h->n),
+                                        cudaMemcpyDeviceToHost, h->s_d2h));
+    }
+  }
+  SGP_CUDA_TRY(h, cudaStreamSynchronize(h->s_h2d));
+  SGP_CUDA_TRY(h, cudaStreamSynchronize(h->s_compute));
+  SGP_CUDA_TRY(h, cudaStreamSynchronize(h->s_d2h));
+  return refresh_status(h, nullptr);
+}
+
 }  // namespace
 
 extern "C" {
@@ -630,61 +709,32 @@ int sgp_debias(sgp_handle *h, const float *d_X, const float *d_W, float *d_Z, vo
 int sgp_step_host(sgp_handle *h, float *d_X, float *d_W, float *d_M, const float *h_G, float *h_Z, float *d_G,
                   float *d_Z, int64_t k, float lr, float momentum, float weight_decay, int nesterov,
                   int64_t chunk_cols, void *stream) {
-  int rc = validate_step(h, d_X, d_W, d_M, d_G, k, momentum);
+  const int rc = validate_step(h, d_X, d_W, d_M, d_G, k, momentum);
   if (rc != SGP_OK) return rc;
   if (h_G == nullptr || (h_Z != nullptr && d_Z == nullptr)) return SGP_ERR_ARG;
-  if (h->seen_status & kWaitBits) return SGP_ERR_DEVICE;
-  if (h->seen_status & sgp::kStatusZeroWeight) return SGP_ERR_ZERO_WEIGHT;
-  if (h->s_h2d == nullptr) {
-    SGP_CUDA_TRY(h, cudaStreamCreateWithFlags(&h->s_h2d, cudaStreamNonBlocking));
-    SGP_CUDA_TRY(h, cudaStreamCreateWithFlags(&h->s_compute, cudaStreamNonBlocking));
-    SGP_CUDA_TRY(h, cudaStreamCreateWithFlags(&h->s_d2h, cudaStreamNonBlocking));
-    SGP_CUDA_TRY(h, cudaEventCreateWithFlags(&h->ev_entry, cudaEventDisableTiming));
-  }
-  // default chunk: about 64 MB of gradient per chunk, a multiple of 1024 columns
-  if (chunk_cols <= 0) chunk_cols = std::max<int64_t>(1024, (int64_t{64} << 20) / (4 * h->n) / 1024 * 1024);
-  chunk_cols = (chunk_cols + 3) / 4 * 4;
-  const int64_t nchunks = (h->d + chunk_cols - 1) / chunk_cols;
-  while (static_cast<int64_t>(h->ev_in.size()) < nchunks) {
-    cudaEvent_t a = nullptr, b = nullptr;
-    SGP_CUDA_TRY(h, cudaEventCreateWithFlags(&a, cudaEventDisableTiming));
-    h->ev_in.push_back(a);
-    SGP_CUDA_TRY(h, cudaEventCreateWithFlags(&b, cudaEventDisableTiming));
-    h->ev_done.push_back(b);
-  }
-  // what the caller already enqueued on its stream (it may produce X, W, M or read d_G, d_Z) comes first:
-  // an event wait on the device, not a host synchronisation
-  SGP_CUDA_TRY(h, cudaEventRecord(h->ev_entry, static_cast<cudaStream_t>(stream)));
-  SGP_CUDA_TRY(h, cudaStreamWaitEvent(h->s_h2d, h->ev_entry, 0));
-  SGP_CUDA_TRY(h, cudaStreamWaitEvent(h->s_compute, h->ev_entry, 0));
-  SGP_CUDA_TRY(h, cudaStreamWaitEvent(h->s_d2h, h->ev_entry, 0));
   const StepArgs a{d_X, d_W, momentum != 0.0f ? d_M : nullptr, d_G, h_Z != nullptr ? d_Z : nullptr,
                    k, lr, momentum, weight_decay, update_kind(momentum, nesterov)};
-  if (h->opt_diagnostics) {
-    SGP_CUDA_TRY(h, cudaMemsetAsync(h->d_stats + kDevStatsDiag, 0, 2 * static_cast<size_t>(h->n) * sizeof(double), h->s_compute));
-    h->diag_valid = true;
-  }
-  const size_t pitch = static_cast<size_t>(h->ld) * sizeof(float);
-  for (int64_t c = 0; c < nchunks; ++c) {
-    const int64_t c0 = c * chunk_cols, c1 = std::min(h->d, c0 + chunk_cols);
-    const size_t width = static_cast<size_t>(c1 - c0) * sizeof(float);
-    SGP_CUDA_TRY(h, cudaMemcpy2DAsync(d_G + c0, pitch, h_G + c0, pitch, width, static_cast<size_t>(h->n),
-                                      cudaMemcpyHostToDevice, h->s_h2d));
-    SGP_CUDA_TRY(h, cudaEventRecord(h->ev_in[static_cast<size_t>(c)], h->s_h2d));
-    SGP_CUDA_TRY(h, cudaStreamWaitEvent(h->s_compute, h->ev_in[static_cast<size_t>(c)], 0));
-    rc = launch_step_range(h, a, c0, c1, c == nchunks - 1, h->s_compute);
-    if (rc != SGP_OK) return rc;
-    if (h_Z != nullptr) {
-      SGP_CUDA_TRY(h, cudaEventRecord(h->ev_done[static_cast<size_t>(c)], h->s_compute));
-      SGP_CUDA_TRY(h, cudaStreamWaitEvent(h->s_d2h, h->ev_done[static_cast<size_t>(c)], 0));
-      SGP_CUDA_TRY(h, cudaMemcpy2DAsync(h_Z + c0, pitch, d_Z + c0, pitch, width, static_cast<size_t>(h->n),
-                                        cudaMemcpyDeviceToHost, h->s_d2h));
-    }
-  }
-  SGP_CUDA_TRY(h, cudaStreamSynchronize(h->s_h2d));
-  SGP_CUDA_TRY(h, cudaStreamSynchronize(h->s_compute));
-  SGP_CUDA_TRY(h, cudaStreamSynchronize(h->s_d2h));
-  return refresh_status(h, nullptr);
+  return run_host_step(h, a, h_G, h_Z, chunk_cols, stream);
+}
+
+int sgp_step_adam_host(sgp_handle *h, float *d_X, float *d_W, float *d_M1, float *d_M2, const float *h_G, float *h_Z,
+                       float *d_G, float *d_Z, int64_t k, int64_t t, float lr, float beta1, float beta2, float eps,
+                       float weight_decay, int64_t chunk_cols, void *stream) {
+  if (h == nullptr || d_X == nullptr || d_W == nullptr || d_M1 == nullptr || d_M2 == nullptr || d_G == nullptr ||
+      h_G == nullptr || (h_Z != nullptr && d_Z == nullptr) || k < 0 || t < 1 || !(beta1 >= 0.0f && beta1 < 1.0f) ||
+      !(beta2 >= 0.0f && beta2 < 1.0f) || !(eps >= 0.0f))
+    return SGP_ERR_ARG;
+  if (check_device(h) != SGP_OK) return check_device(h);
+  StepArgs a{d_X, d_W, d_M1, d_G, h_Z != nullptr ? d_Z : nullptr, k, lr, 0.0f, weight_decay, sgp::kUpdAdam};
+  a.V = d_M2;
+  a.beta1 = beta1;
+  a.beta2 = beta2;
+  a.eps = eps;
+  const double bc1 = 1.0 - std::pow(static_cast<double>(beta1), static_cast<double>(t));
+  const double bc2 = 1.0 - std::pow(static_cast<double>(beta2), static_cast<double>(t));
+  a.adam_step = static_cast<float>(static_cast<double>(lr) / bc1);
+  a.adam_rsqrt_bc2 = static_cast<float>(1.0 / std::sqrt(bc2));
+  return run_host_step(h, a, h_G, h_Z, chunk_cols, stream);
 }
 
 int sgp_reset(sgp_handle *h, void *stream) {
@@ -821,8 +871,11 @@ int sgp_param_deviation(sgp_handle *h, const float *d_A, double *h_dev, void *st
 int sgp_set_option(sgp_handle *h, const char *key, int64_t value) {
   if (h == nullptr || key == nullptr || value < 0) return SGP_ERR_ARG;
   if (std::strcmp(key, "variant") == 0) {
-    if (value > 3) return SGP_ERR_ARG;
+    if (value > 4) return SGP_ERR_ARG;
     h->opt_variant = value;
+  } else if (std::strcmp(key, "cluster") == 0) {
+    if (value != 0 && value != 1 && value != 2 && value != 4) return SGP_ERR_ARG;
+    h->opt_cluster = value;
   } else if (std::strcmp(key, "tile_cols") == 0) {
     if (value % 4 != 0 || value > 4096) return SGP_ERR_ARG;
     h->opt_tile_cols = value;
@@ -878,6 +931,7 @@ int sgp_get_option(const sgp_handle *h, const char *key, int64_t *value) {
   else if (std::strcmp(key, "wait_limit_ms") == 0) *value = h->opt_wait_limit_ms;
   else if (std::strcmp(key, "inject_stall") == 0) *value = h->opt_inject_stall;
   else if (std::strcmp(key, "send_period") == 0) *value = h->opt_send_period;
+  else if (std::strcmp(key, "cluster") == 0) *value = h->opt_cluster;
   else if (std::strcmp(key, "diagnostics") == 0) *value = h->opt_diagnostics;
   else if (std::strcmp(key, "check_steps") == 0) *value = h->opt_check_steps;
   else if (std::strcmp(key, "last_variant") == 0) *value = h->last.variant;

@@ -132,3 +132,31 @@ def test_adam_argument_checks(binding):
         assert ok(b1=1.0) == binding.SGP_ERR_ARG
         assert ok(m2=None) == binding.SGP_ERR_ARG
         torch.cuda.synchronize()
+
+
+def test_adam_step_host_matches_device_step(binding, inputs):
+    """Host-buffer entry point for Adam-SGP: bit-identical to the device step (columns are independent, chunks too)."""
+    import dataclasses
+    w = dataclasses.replace(inputs.WORKLOADS["transformer_adam"].scaled(40_003, K=3), tau=1)
+    n, d = w.n, w.d
+    def state():
+        X = inputs.initial_x(w, device=DEV).contiguous()
+        return X, torch.ones(n, device=DEV), torch.zeros_like(X), torch.zeros_like(X), torch.empty_like(X)
+    Xa, Wa, M1a, M2a, Za = state()
+    Xb, Wb, M1b, M2b, Zb = state()
+    G = torch.empty((n, d), device=DEV)
+    hG = torch.empty((n, d), pin_memory=True)
+    hZ = torch.empty((n, d), pin_memory=True)
+    dG = torch.empty((n, d), device=DEV)
+    with binding.Sgp(n, d, graph_desc(w, binding), tau=1) as h1, binding.Sgp(n, d, graph_desc(w, binding), tau=1) as h2:
+        for k in range(3):
+            inputs.gradient(w, k, G)
+            hG.copy_(G)
+            torch.cuda.synchronize()
+            h1.step_adam(Xa, Wa, M1a, M2a, G, Za, k, k + 1, w.lr, w.beta1, w.beta2, w.adam_eps, 1e-3)
+            h2.step_adam_host(Xb, Wb, M1b, M2b, hG, hZ, dG, Zb, k, k + 1, w.lr, w.beta1, w.beta2, w.adam_eps, 1e-3,
+                              chunk_cols=8192)
+        torch.cuda.synchronize()
+    for a, b in ((Xa, Xb), (Wa, Wb), (M1a, M1b), (M2a, M2b), (Za, Zb)):
+        assert torch.equal(a, b)
+    assert torch.equal(hZ.to(DEV), Za)

@@ -2,6 +2,7 @@
 on the same seeded inputs.  Sizes span several column tiles and a ragged tail; the w != 1 cases
 (irregular graphs, delayed messages) are included because regular graphs cannot detect a broken
 weight path."""
+import dataclasses
 from fractions import Fraction
 
 import numpy as np
@@ -455,3 +456,37 @@ def test_complete_graph_shared_column_sum_path(binding, inputs, n, d, variant):
     out = _run_gpu(binding, inputs, w, options={"variant": variant})
     _compare(w, out)
     assert np.abs(out["Z"] - out["Z"][0]).max() == 0.0               # every node holds the same vector, bit for bit
+
+
+# ------------------------------------------------------------------ thread-block-cluster kernel (many nodes)
+@pytest.mark.parametrize("n,d,tau,cluster", [(256, 1_029, 0, 4), (256, 4_100, 1, 4), (200, 3_001, 0, 4), (130, 2_052, 2, 4),
+                                             (129, 1_500, 0, 2), (64, 9_000, 0, 2), (5, 2_000, 1, 4), (2, 700, 0, 2),
+                                             (256, 70_001, 0, 4), (3, 1_000, 0, 4)])
+def test_cluster_kernel_matches_oracle_and_register_kernel(binding, inputs, n, d, tau, cluster):
+    """A cluster of CTAs holds the tile's rows together and gathers through distributed shared memory: same CSR
+    order and FMA chain as the one-CTA kernels, so results are bit-identical to theirs and within tolerance of the
+    oracle.  n = 3 with four CTAs leaves one CTA without rows; n = 200 leaves the last CTA a partial slice."""
+    w = dataclasses.replace(inputs.sweep_workload(n, d), tau=tau, weight_decay=1e-3, K=5)
+    a = _run_gpu(binding, inputs, w, options={"variant": 4, "cluster": cluster})
+    _compare(w, a)
+    b = _run_gpu(binding, inputs, w, options={"variant": 1})
+    for name in ("X", "Z", "M", "W"):
+        assert np.array_equal(a[name], b[name]), name
+
+
+def test_cluster_kernel_is_opt_in(binding, inputs):
+    w = inputs.sweep_workload(256, 300_000)
+    X = inputs.initial_x(w, device=DEV).contiguous()
+    W = torch.ones(w.n, device=DEV); M = torch.zeros_like(X); Z = torch.empty_like(X)
+    G = inputs.gradient(w, 0, torch.empty_like(X))
+    with binding.Sgp(w.n, w.d, graph_desc(w, binding)) as h:
+        h.step(X, W, M, G, Z, 0, w.lr, w.momentum, 0.0, True)
+        torch.cuda.synchronize()
+        assert h.get_option("last_variant") == 1
+        h.set_option("variant", 4)
+        h.set_option("cluster", 4)
+        h.step(X, W, M, G, Z, 1, w.lr, w.momentum, 0.0, True)
+        torch.cuda.synchronize()
+        assert h.get_option("last_variant") == 4 and h.get_option("last_tile_cols") == 256
+        assert h.get_option("last_grid") % 4 == 0
+        assert h.device_status() == 0
