@@ -900,6 +900,17 @@ int sgp_set_option(sgp_handle *h, const char *key, int64_t value) {
   } else if (std::strcmp(key, "send_period") == 0) {
     if (value < 1 || value > (1 << 20)) return SGP_ERR_ARG;
     h->opt_send_period = value;
+#ifdef SGP_CHECKED
+  } else if (std::strcmp(key, "poke_table") == 0) {
+    // Bounds-checked build only, test hook: overwrites the first sender index of slot 0's table with `value`, so that
+    // a test can watch an out-of-range index being caught (status bit, access skipped) instead of dereferenced.
+    const int32_t bad = static_cast<int32_t>(value);
+    if (cudaMemcpy(h->d_col + h->off_nnz[0], &bad, sizeof(bad), cudaMemcpyHostToDevice) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return SGP_ERR_CUDA;
+    }
+    if (h->const_ok[0]) h->const_tables[0].col[0] = bad;
+#endif
   } else if (std::strcmp(key, "diagnostics") == 0) {
     if (value > 1) return SGP_ERR_ARG;
     h->opt_diagnostics = value;
