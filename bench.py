@@ -536,7 +536,8 @@ def main():
     ap.add_argument("--arm", default="sgp", choices=["sgp", "osgp", "allreduce"], help="--mode rowshard only")
     ap.add_argument("--d", type=int, default=0, help="override the parameter count (profiling on a small case)")
     ap.add_argument("--n", type=int, default=0, help="override the node count (rowshard-loopback)")
-    ap.add_argument("--tau", type=int, default=-1, help="override the delay (rowshard-loopback)")
+    ap.add_argument("--tau", type=int, default=-1, help="override the delay")
+    ap.add_argument("--peers", type=int, default=0, help="override the out-neighbours per node of the exponential graph")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--option", action="append", default=[], help="key=value passed to sgp_set_option")
@@ -562,6 +563,8 @@ def main():
         w = dataclasses.replace(w, n=args.n)
     if args.tau >= 0:
         w = dataclasses.replace(w, tau=args.tau)
+    if args.peers > 0:
+        w = dataclasses.replace(w, peers=args.peers)
     if args.impl == "reference":
         run_reference(args, w)
         return

@@ -231,6 +231,7 @@ sgp_step_tma_kernel(const __grid_constant__ StepParams p, const __grid_constant_
       const float4 *Rs = Xs + static_cast<size_t>(kIdxR) * tile_items;
       // phase 1: local update; x^(k+1/2) replaces x in the stage
       float4 csum = make_float4(0.f, 0.f, 0.f, 0.f), rsum = csum;   // diagnostics: this thread's share of its column's sums
+#pragma unroll 4
       for (int item = ctid; item < tile_items; item += kTmaConsumers) {
         const int row = item >> p.log2_tile_vecs;
         const int c = item & (tv - 1);
@@ -295,35 +296,61 @@ sgp_step_tma_kernel(const __grid_constant__ StepParams p, const __grid_constant_
         if (lane == 0) mbar_arrive(empty_bar + s);
         continue;
       }
-      // phase 2: gather-mix, ring exchange, de-bias
-      for (int item = ctid; item < tile_items; item += kTmaConsumers) {
-        const int row = item >> p.log2_tile_vecs;
-        const int c = item & (tv - 1);
-        const int64_t col = col0 + static_cast<int64_t>(c) * 4;
-        if (col < p.col_end) {
-          const int64_t o = static_cast<int64_t>(row) * ld + col;
-          float4 acc = make_float4(0.f, 0.f, 0.f, 0.f), offd = acc;
-          const int e1 = tab.rowptr[row + 1];
-          for (int e = tab.rowptr[row]; e < e1; ++e) {
-            const int j = tab.col[e];
-            if (!SGP_BOUNDS_OK(p, j >= 0 && j < n)) continue;
-            const float pv = tab.val[e];
-            const float4 hj = Xs[(j << p.log2_tile_vecs) + c];
-            if (HAS_RING && j != row) offd = vfma(pv, hj, offd);
-            else acc = vfma(pv, hj, acc);
+      // phase 2: gather-mix, ring exchange, de-bias.  A thread works on kGather of its items at once: their
+      // in-neighbour lists are walked together, so that kGather independent shared-memory loads and FMA chains are
+      // in flight instead of one (the eight consumer warps are all the latency hiding this kernel has).
+      constexpr int kGather = 4;
+      for (int it0 = ctid; it0 < tile_items; it0 += kGather * kTmaConsumers) {
+        int e0[kGather], len[kGather], cc[kGather];
+        bool act[kGather];
+        float4 acc[kGather], offd[kGather];
+        int maxlen = 0;
+#pragma unroll
+        for (int q = 0; q < kGather; ++q) {
+          const int item = it0 + q * kTmaConsumers;
+          const int row = item >> p.log2_tile_vecs;
+          cc[q] = item & (tv - 1);
+          act[q] = item < tile_items && col0 + static_cast<int64_t>(cc[q]) * 4 < p.col_end;
+          e0[q] = act[q] ? tab.rowptr[row] : 0;
+          len[q] = act[q] ? tab.rowptr[row + 1] - e0[q] : 0;
+          maxlen = max(maxlen, len[q]);
+          acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+          offd[q] = acc[q];
+        }
+        for (int e = 0; e < maxlen; ++e) {
+#pragma unroll
+          for (int q = 0; q < kGather; ++q) {
+            if (e < len[q]) {
+              const int j = tab.col[e0[q] + e];
+              if (SGP_BOUNDS_OK(p, j >= 0 && j < n)) {
+                const float pv = tab.val[e0[q] + e];
+                const float4 hj = Xs[(j << p.log2_tile_vecs) + cc[q]];
+                if (HAS_RING && j != ((it0 + q * kTmaConsumers) >> p.log2_tile_vecs)) offd[q] = vfma(pv, hj, offd[q]);
+                else acc[q] = vfma(pv, hj, acc[q]);
+              }
+            }
           }
-          if (HAS_RING) {
-            acc = vadd(acc, Rs[item]);
-            st_stream(reinterpret_cast<float4 *>(p.ring_x + o), offd);
-          }
-          const float4 z = vmul(tab.inv_w[row], acc);
-          st_stream(reinterpret_cast<float4 *>(p.X + o), acc);
-          if (HAS_Z) st_stream(reinterpret_cast<float4 *>(p.Z + o), z);
-          if (DIAG) {
-            float2 sq = ds.slots[item];
-            sq.x += vsq(vsub(Xs[item], mean_h));
-            sq.y += vsq(vsub(z, mean_x));
-            ds.slots[item] = sq;
+        }
+#pragma unroll
+        for (int q = 0; q < kGather; ++q) {
+          if (act[q]) {
+            const int item = it0 + q * kTmaConsumers;
+            const int row = item >> p.log2_tile_vecs;
+            const int64_t o = static_cast<int64_t>(row) * ld + col0 + static_cast<int64_t>(cc[q]) * 4;
+            float4 a = acc[q];
+            if (HAS_RING) {
+              a = vadd(a, Rs[item]);
+              st_stream(reinterpret_cast<float4 *>(p.ring_x + o), offd[q]);
+            }
+            const float4 z = vmul(tab.inv_w[row], a);
+            st_stream(reinterpret_cast<float4 *>(p.X + o), a);
+            if (HAS_Z) st_stream(reinterpret_cast<float4 *>(p.Z + o), z);
+            if (DIAG) {
+              float2 sq = ds.slots[item];
+              sq.x += vsq(vsub(Xs[item], mean_h));
+              sq.y += vsq(vsub(z, mean_x));
+              ds.slots[item] = sq;
+            }
           }
         }
       }
