@@ -139,16 +139,15 @@ template <int UPD> struct UpdTraits {
 struct UpdateScalars {
   float lr, momentum, wd, beta1, beta2, eps, adam_step, adam_rsqrt_bc2;
 };
-__device__ __forceinline__ UpdateScalars update_scalars(const StepParams &p) {
-  return UpdateScalars{p.lr, p.momentum, p.wd, p.beta1, p.beta2, p.eps, p.adam_step, p.adam_rsqrt_bc2};
-}
 
 // Local update of one element group: returns h = x^(k+1/2) and updates the optimiser state in place.
 // SGD: Alg. 1 line 4.  Momentum / Nesterov: Alg. 3 lines 4-5.  Adam (Sec. 6.2, App. C.1: Adam-preconditioned
 // SGP): bias-corrected Adam step on the numerator, moments stay local.
 // Weight decay adds wd * x to the gradient in every case.
-template <int UPD, typename V>
-__device__ __forceinline__ V local_update(V x, V g, V &u, V &v, const UpdateScalars &p) {
+// `p` is anything with the fields lr, momentum, wd, beta1, beta2, eps, adam_step, adam_rsqrt_bc2 (StepParams itself,
+// so that the scalars stay constant-bank operands, or UpdateScalars).
+template <int UPD, typename V, typename P>
+__device__ __forceinline__ V local_update(V x, V g, V &u, V &v, const P &p) {
   const V gt = vfma(p.wd, x, g);
   if (UPD == kUpdAdam) {
     u = vfma(p.beta1, u, vmul(1.0f - p.beta1, gt));
@@ -163,10 +162,6 @@ __device__ __forceinline__ V local_update(V x, V g, V &u, V &v, const UpdateScal
     s = UPD == kUpdNesterov ? vfma(p.momentum, u, gt) : u;
   }
   return vfma(-p.lr, s, x);
-}
-template <int UPD, typename V>
-__device__ __forceinline__ V local_update(V x, V g, V &u, V &v, const StepParams &p) {
-  return local_update<UPD, V>(x, g, u, v, update_scalars(p));
 }
 
 // Per-CTA scratch after the tiles/stages in dynamic shared memory: [w_old n][rw_in n][inv_w n], then the

@@ -181,6 +181,51 @@ def test_handle_calls_reject_null_without_a_gpu(binding):
     assert out.value is None
 
 
+def test_new_entry_points_reject_null_without_a_gpu(binding):
+    lib = binding.lib()
+    stats = (C.c_double * 8)()
+    assert lib.sgp_check(None, None, None, None, stats, None) == binding.SGP_ERR_ARG
+    assert lib.sgp_colsum(None, None, 0, None, None) == binding.SGP_ERR_ARG
+    assert lib.sgp_get_diagnostics(None, None, None, None, None) == binding.SGP_ERR_ARG
+    assert lib.sgp_step_adam_host(None, None, None, None, None, None, None, None, None, 0, 1, 0.1, 0.9, 0.99, 1e-8, 0.0, 0,
+                                  None) == binding.SGP_ERR_ARG
+    assert lib.sgp_rank_update(None, None, None, None, None, 0, 0.1, 0.0, 0.0, 1, None) == binding.SGP_ERR_ARG
+    assert lib.sgp_rank_mix(None, None, None, None, 0, None) == binding.SGP_ERR_ARG
+    assert lib.sgp_rank_step_overlap(None, None, None, None, None, None, 0, 0.1, 0.0, 0.0, 1, None) == binding.SGP_ERR_ARG
+    assert lib.sgp_rank_destroy(None) == binding.SGP_OK
+    assert lib.sgp_ipc_export(None, None) == binding.SGP_ERR_ARG and lib.sgp_ipc_close(None) == binding.SGP_OK
+    out = C.c_void_p()
+    g = binding.GraphDesc.exp_peers(1)
+    assert lib.sgp_rank_create(C.byref(out), 4, 4, 100, C.byref(g.c), 0, 0) == binding.SGP_ERR_ARG       # rank == world
+    assert lib.sgp_rank_create(C.byref(out), 0, 4, 100, C.byref(g.c), 0, 8) == binding.SGP_ERR_ARG       # unknown flag
+    assert out.value is None
+    for code, word in ((binding.SGP_ERR_ZERO_WEIGHT, "weight"), (binding.SGP_ERR_INVARIANT, "invariant"),
+                       (binding.SGP_ERR_DEVICE, "wait")):
+        assert word in binding.strerror(code)
+
+
+def test_rank_plan_host_only(binding):
+    """sgp_rank_plan needs no GPU: slots, self weight and the in-neighbour list in the order of the sum."""
+    sched = binding.Schedule(8, binding.GraphDesc.exp_peers(2))
+    for k in range(7):
+        P = S.mixing_matrix("exp", 8, k, peers=2)
+        for r in range(8):
+            plan = binding.rank_plan(sched, r, k, 0)
+            want = [j for j in range(8) if P[r, j] != 0.0]
+            assert plan["senders"] == want and plan["self_pos"] == want.index(r)
+            assert plan["write_slot"] == plan["read_slot"] == k % 2
+            assert np.array_equal(plan["weights"], np.array([P[r, j] for j in want], dtype=np.float32))
+            late = binding.rank_plan(sched, r, k, 3)
+            Pd = S.mixing_matrix("exp", 8, k - 3, peers=2) if k >= 3 else np.zeros((8, 8))
+            assert late["senders"] == [j for j in range(8) if Pd[r, j] != 0.0 and j != r]
+            assert late["write_slot"] == k % 5 and late["read_slot"] == (k - 3) % 5 and late["self_pos"] == -1
+            assert late["self_weight"] == np.float32(P[r, r])
+    for bad in ((8, 0, 0), (-1, 0, 0), (0, -1, 0), (0, 0, -1), (0, 0, 65)):
+        with pytest.raises(binding.SgpError) as e:
+            binding.rank_plan(sched, *bad)
+        assert e.value.code == binding.SGP_ERR_ARG
+
+
 def _random_custom_schedule(n, steps, seed):
     """Random column-stochastic schedule with NON-uniform fp32 weights (every column sums to 1 in fp32 exactly
     enough for the compiler's check): per sender a random out-set incl. self and Dirichlet-like weights."""
