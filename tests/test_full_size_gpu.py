@@ -161,3 +161,48 @@ def test_tau_full_size_mass_conservation(binding, inputs):
         stats = h.check(X, W, colsum_ref=ref)
     assert stats["code"] == 0 and stats["max_colsum_rel_drift"] <= 2e-6, stats
     assert abs(stats["sum_w"] - n) <= 1e-4 * n and stats["nonfinite"] == 0
+
+
+@pytest.mark.parametrize("name", ["resnet50", "resnet50_osgp1"])
+def test_fused_diagnostics_full_size(binding, inputs, name):
+    """The diagnostics of the full-size launch (every CTA accumulates hundreds of tiles in fp32 slots) against the same
+    quantities formed from the arrays with float64 torch arithmetic on the device: properties that hold at any size.
+    Parameter deviation (Sec. 6.1): || h_i - mean_j h_j || with h = x - lr (m u' + g + wd x) rebuilt from the state
+    before the step and the momentum after it; consensus distance: || z_i - xbar ||, xbar = (colsum(X') + ring') / n."""
+    w = inputs.WORKLOADS[name]
+    n, d = w.n, w.d
+    X, ld = binding.empty_matrix(n, d, device=DEV)
+    X.copy_(inputs.initial_x(w, device=DEV))
+    M, _ = binding.empty_matrix(n, d, device=DEV, fill=0.0)
+    Z, _ = binding.empty_matrix(n, d, device=DEV, fill=float("nan"))
+    G, _ = binding.empty_matrix(n, d, device=DEV)
+    W = torch.ones(n, device=DEV)
+    with binding.Sgp(n, d, binding.graph_desc(w), tau=w.tau, ld=ld) as h:
+        for k in range(3):
+            inputs.gradient(w, k, G)
+            X += 0.01 * torch.arange(n, device=DEV, dtype=torch.float32)[:, None] if k == 0 else 0.0   # nodes differ
+            if k == 2:
+                h.set_option("diagnostics", 1)
+                X_before = X.clone()
+            h.step(X, W, M, G, Z, k, w.lr, w.momentum, w.weight_decay, True)
+        dev, cons, summary = h.diagnostics()
+        colsum_after = h.colsum(X, include_ring=True)
+        assert h.device_status() == 0
+    lr, m, wd = (float(np.float32(v)) for v in (w.lr, w.momentum, w.weight_decay))
+    want_dev = torch.zeros(n, dtype=torch.float64, device=DEV)
+    want_cons = torch.zeros(n, dtype=torch.float64, device=DEV)
+    step = 1 << 21
+    for c0 in range(0, d, step):
+        c1 = min(d, c0 + step)
+        xb, g, mu = X_before[:, c0:c1].double(), G[:, c0:c1].double(), M[:, c0:c1].double()
+        hh = xb - lr * (m * mu + g + wd * xb)
+        want_dev += ((hh - hh.mean(dim=0, keepdim=True)) ** 2).sum(dim=1)
+        xbar = colsum_after[c0:c1] / n
+        want_cons += ((Z[:, c0:c1].double() - xbar[None, :]) ** 2).sum(dim=1)
+    want_dev, want_cons = want_dev.sqrt().cpu().numpy(), want_cons.sqrt().cpu().numpy()
+    assert np.abs(dev - want_dev).max() <= 2e-5 * want_dev.max(), (dev[:4], want_dev[:4])
+    assert np.abs(cons - want_cons).max() <= 2e-5 * max(want_cons.max(), want_dev.max()), (cons[:4], want_cons[:4])
+    assert abs(summary["param_dev_max"] - want_dev.max()) <= 2e-5 * want_dev.max()
+    assert want_dev.min() > 0
+    del X, M, Z, G, X_before
+    torch.cuda.empty_cache()
