@@ -1,6 +1,7 @@
 // C ABI of the fused SGP step (see include/sgp.h): handle management, argument validation, launch
 // plan and dispatch.  All arithmetic of the method lives in the kernels.
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 
 #include <algorithm>
 #include <cmath>
@@ -80,6 +81,14 @@ namespace {
   } while (0)
 
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// NVTX range around an entry point's host work (header-only NVTX: a no-op unless a tool is attached).
+struct NvtxRange {
+  explicit NvtxRange(const char *name) { nvtxRangePushA(name); }
+  ~NvtxRange() { nvtxRangePop(); }
+  NvtxRange(const NvtxRange &) = delete;
+  NvtxRange &operator=(const NvtxRange &) = delete;
+};
 
 void free_handle(sgp_handle *h) {
   if (h == nullptr) return;
@@ -405,6 +414,7 @@ int enqueue_check(sgp_handle *h, const float *X, const float *W, const double *r
 
 // A whole step on the device arrays: optional debug bracket, optional diagnostics, the fused launch(es).
 int run_step(sgp_handle *h, const StepArgs &a, cudaStream_t st) {
+  const NvtxRange range(a.upd == sgp::kUpdAdam ? "sgp_step_adam" : "sgp_step");
   if (h->seen_status & kWaitBits) return SGP_ERR_DEVICE;
   if (h->seen_status & sgp::kStatusZeroWeight) return SGP_ERR_ZERO_WEIGHT;
   if (h->opt_check_steps) {
@@ -513,6 +523,7 @@ int refresh_status(sgp_handle *h, unsigned *out) {
 // The host-buffer step: column chunks pipelined over three streams (H2D of chunk c+1, fused step on chunk c, D2H of
 // chunk c-1); `a` carries the device arrays and the optimiser, a.G / a.Z are the device staging arrays.
 int run_host_step(sgp_handle *h, const StepArgs &a, const float *h_G, float *h_Z, int64_t chunk_cols, void *stream) {
+  const NvtxRange range("sgp_step_host");
   float *d_G = const_cast<float *>(a.G);
   float *d_Z = a.Z;
   int rc = SGP_OK;
@@ -788,6 +799,7 @@ int sgp_colsum(sgp_handle *h, const float *d_A, int include_ring, double *d_out,
 int sgp_check(sgp_handle *h, const float *d_X, const float *d_W, const double *d_colsum_ref, double *h_stats,
               void *stream) {
   if (h == nullptr || d_X == nullptr || d_W == nullptr || h_stats == nullptr) return SGP_ERR_ARG;
+  const NvtxRange range("sgp_check");
   int rc = check_device(h);
   if (rc != SGP_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
