@@ -14,6 +14,7 @@ import numpy as np
 _PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 # SGP_CHECKED=1 in the environment selects the bounds-checked build of the same library (build.build_checked()).
 LIB_PATH = os.path.join(_PKG_DIR, "libsgp_checked.so" if os.environ.get("SGP_CHECKED", "0") not in ("", "0") else "libsgp.so")
+LIB_PATH = os.environ.get("SGP_LIBRARY", LIB_PATH)          # an explicit path wins (another build of the same sources)
 
 SGP_OK, SGP_ERR_ARG, SGP_ERR_GRAPH, SGP_ERR_CUDA, SGP_ERR_ALLOC, SGP_ERR_STATE, SGP_ERR_DEVICE = 0, -1, -2, -3, -4, -5, -6
 SGP_ERR_ZERO_WEIGHT, SGP_ERR_INVARIANT = -7, -8

@@ -221,6 +221,9 @@ Plan make_plan(const sgp_handle *h, int arrays, bool has_m, int nnz, bool vec) {
       pl.tile_cols = sgp::regs_tile_cols(h->n, fixed);
     }
   }
+  // Diagnostics with a momentum update: the register-staged instantiation carries them for free (n = 32: 0.971 of the
+  // copy bandwidth with them, 0.955 without; the pipelined kernel 0.964 with them).
+  if (vec && h->opt_diagnostics && has_m && pl.variant >= 2) pl = Plan{1, sgp::regs_tile_cols(h->n, 4 * 1024), 2, 0};
   if (h->opt_variant > 0 && (h->opt_variant == 1) != (pl.variant == 1)) {
     // the caller forces the other kernel family: take that family's defaults
     if (h->opt_variant == 1 || h->opt_variant == 4) {
