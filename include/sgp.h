@@ -350,7 +350,7 @@ int sgp_step_static(int n, int64_t d, int64_t ld, const int32_t *h_rowptr, const
  * step's stream): tau == 0: update, BARRIER, mix; tau >= 1: step_overlap, BARRIER.  No kernel of this library
  * waits on another GPU.  A rank keeps tau + 2 message slots: a slot is rewritten tau + 2 steps after it was
  * published, when every reader has passed at least one barrier since its read.
- * Not supported here: send_period, Adam, in-degree above SGP_RANK_MAX_SOURCES (SGP_ERR_ARG; the complete graph
+ * Not supported here: send_period, in-degree above SGP_RANK_MAX_SOURCES (SGP_ERR_ARG; the complete graph
  * is what an all-reduce is for).
  * ------------------------------------------------------------------------------------------- */
 typedef struct sgp_rank sgp_rank;
@@ -393,6 +393,13 @@ int sgp_rank_mix(sgp_rank *r, float *d_x, float *d_w, float *d_z, int64_t k, voi
  * tau == 0.  Asynchronous. */
 int sgp_rank_step_overlap(sgp_rank *r, float *d_x, float *d_w, float *d_m, const float *d_g, float *d_z, int64_t k,
                           float lr, float momentum, float weight_decay, int nesterov, void *stream);
+/* The same two calls with the Adam preconditioner (Sec. 6.2 / App. C.1; arguments as sgp_step_adam: t >= 1 counts
+ * the Adam steps including this one; m1, m2 are this node's moment rows, never sent). */
+int sgp_rank_update_adam(sgp_rank *r, const float *d_x, float *d_w, float *d_m1, float *d_m2, const float *d_g, int64_t k,
+                         int64_t t, float lr, float beta1, float beta2, float eps, float weight_decay, void *stream);
+int sgp_rank_step_overlap_adam(sgp_rank *r, float *d_x, float *d_w, float *d_m1, float *d_m2, const float *d_g, float *d_z,
+                               int64_t k, int64_t t, float lr, float beta1, float beta2, float eps, float weight_decay,
+                               void *stream);
 /* SGP_STATUS_ZERO_WEIGHT is the only bit this mode sets.  Synchronises. */
 int sgp_rank_device_status(sgp_rank *r, unsigned *status);
 /* Thin wrappers of the CUDA IPC calls for callers without a CUDA binding: `handle` is SGP_IPC_HANDLE_BYTES bytes of

@@ -34,7 +34,8 @@ EXPORTS = [
     "sgp_step_adam", "sgp_param_deviation", "sgp_set_graph", "sgp_colsum", "sgp_get_diagnostics",
     "sgp_rank_plan", "sgp_rank_create", "sgp_rank_destroy", "sgp_rank_get_schedule", "sgp_rank_message_block",
     "sgp_rank_set_peers", "sgp_rank_update", "sgp_rank_mix", "sgp_rank_step_overlap", "sgp_rank_device_status",
-    "sgp_ipc_export", "sgp_ipc_open", "sgp_ipc_close", "sgp_step_adam_host",
+    "sgp_ipc_export", "sgp_ipc_open", "sgp_ipc_close", "sgp_step_adam_host", "sgp_rank_update_adam",
+    "sgp_rank_step_overlap_adam",
 ]
 SGP_RANK_MAX_SOURCES = 32
 SGP_IPC_HANDLE_BYTES = 64
@@ -104,6 +105,8 @@ def _load() -> C.CDLL:
         "sgp_rank_update": [vp, vp, vp, vp, vp, i64, f32, f32, f32, i32, vp],
         "sgp_rank_mix": [vp, vp, vp, vp, i64, vp],
         "sgp_rank_step_overlap": [vp, vp, vp, vp, vp, vp, i64, f32, f32, f32, i32, vp],
+        "sgp_rank_update_adam": [vp, vp, vp, vp, vp, vp, i64, i64, f32, f32, f32, f32, f32, vp],
+        "sgp_rank_step_overlap_adam": [vp, vp, vp, vp, vp, vp, vp, i64, i64, f32, f32, f32, f32, f32, vp],
         "sgp_rank_device_status": [vp, C.POINTER(C.c_uint)],
         "sgp_ipc_export": [vp, C.c_char_p],
         "sgp_ipc_open": [C.c_char_p, C.POINTER(vp)],
@@ -438,6 +441,17 @@ class SgpRank:
         _check(_lib.sgp_rank_step_overlap(self._h, _ptr(x), _ptr(w), _ptr(m), _ptr(g), _ptr(z), k, lr, momentum,
                                           weight_decay, int(bool(nesterov)), _stream_ptr(stream)),
                "sgp_rank_step_overlap")
+
+    def update_adam(self, x, w, m1, m2, g, k: int, t: int, lr: float, beta1: float = 0.9, beta2: float = 0.999,
+                    eps: float = 1e-8, weight_decay: float = 0.0, stream=None) -> None:
+        _check(_lib.sgp_rank_update_adam(self._h, _ptr(x), _ptr(w), _ptr(m1), _ptr(m2), _ptr(g), k, t, lr, beta1, beta2,
+                                         eps, weight_decay, _stream_ptr(stream)), "sgp_rank_update_adam")
+
+    def step_overlap_adam(self, x, w, m1, m2, g, z, k: int, t: int, lr: float, beta1: float = 0.9, beta2: float = 0.999,
+                          eps: float = 1e-8, weight_decay: float = 0.0, stream=None) -> None:
+        _check(_lib.sgp_rank_step_overlap_adam(self._h, _ptr(x), _ptr(w), _ptr(m1), _ptr(m2), _ptr(g), _ptr(z), k, t, lr,
+                                               beta1, beta2, eps, weight_decay, _stream_ptr(stream)),
+               "sgp_rank_step_overlap_adam")
 
     def device_status(self) -> int:
         v = C.c_uint()

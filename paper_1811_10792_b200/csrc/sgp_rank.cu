@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <cmath>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -205,34 +206,112 @@ int sgp_rank_get_schedule(const sgp_rank *r, const sgp_schedule **s) {
   return SGP_OK;
 }
 
-int sgp_rank_update(sgp_rank *r, const float *d_x, float *d_w, float *d_m, const float *d_g, int64_t k, float lr,
-                    float momentum, float weight_decay, int nesterov, void *stream) {
-  if (r == nullptr || d_x == nullptr || d_w == nullptr || d_g == nullptr || k < 0 || (momentum != 0.0f && d_m == nullptr))
-    return SGP_ERR_ARG;
+}  // extern "C"
+
+namespace {
+
+sgp::UpdateScalars adam_scalars(float lr, float beta1, float beta2, float eps, float weight_decay, int64_t t) {
+  // bias corrections in double, rounded once (t >= 1), as in the stacked Adam step
+  const double bc1 = 1.0 - std::pow(static_cast<double>(beta1), static_cast<double>(t));
+  const double bc2 = 1.0 - std::pow(static_cast<double>(beta2), static_cast<double>(t));
+  return sgp::UpdateScalars{lr, 0.0f, weight_decay, beta1, beta2, eps, static_cast<float>(static_cast<double>(lr) / bc1),
+                            static_cast<float>(1.0 / std::sqrt(bc2))};
+}
+
+bool adam_args_ok(int64_t t, float beta1, float beta2, float eps) {
+  return t >= 1 && beta1 >= 0.0f && beta1 < 1.0f && beta2 >= 0.0f && beta2 < 1.0f && eps >= 0.0f;
+}
+
+int rank_update(sgp_rank *r, const float *d_x, float *d_w, float *d_m, float *d_v, const float *d_g, int64_t k, int upd,
+                const sgp::UpdateScalars &us, void *stream) {
   int rc = check_device(r);
   if (rc != SGP_OK) return rc;
   sgp::RankParams p{};
   fill_params(r, &p);
   p.x = const_cast<float *>(d_x);
   p.w = d_w;
-  p.m = momentum != 0.0f ? d_m : nullptr;
+  p.m = d_m;
+  p.v = d_v;
   p.g = d_g;
   p.msg = r->block + (k % r->slots) * r->slot_floats;
-  p.us = sgp::UpdateScalars{lr, momentum, weight_decay, 0.f, 0.f, 0.f, 0.f, 0.f};
-  const bool vec = aligned16(d_x) && aligned16(d_g) && (p.m == nullptr || aligned16(p.m));
+  p.us = us;
+  const bool vec = aligned16(d_x) && aligned16(d_g) && (d_m == nullptr || aligned16(d_m)) && (d_v == nullptr || aligned16(d_v));
   const unsigned grid = stream_grid(r, vec);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const int upd = update_kind(momentum, nesterov);
 #define SGP_LAUNCH_UPDATE(VEC)                                                                                   \
   switch (upd) {                                                                                                 \
     case sgp::kUpdSgd: sgp::sgp_rank_update_kernel<VEC, sgp::kUpdSgd><<<grid, sgp::kRankThreads, 0, st>>>(p); break; \
     case sgp::kUpdHeavyBall: sgp::sgp_rank_update_kernel<VEC, sgp::kUpdHeavyBall><<<grid, sgp::kRankThreads, 0, st>>>(p); break; \
-    default: sgp::sgp_rank_update_kernel<VEC, sgp::kUpdNesterov><<<grid, sgp::kRankThreads, 0, st>>>(p);          \
+    case sgp::kUpdNesterov: sgp::sgp_rank_update_kernel<VEC, sgp::kUpdNesterov><<<grid, sgp::kRankThreads, 0, st>>>(p); break; \
+    default: sgp::sgp_rank_update_kernel<VEC, sgp::kUpdAdam><<<grid, sgp::kRankThreads, 0, st>>>(p);              \
   }
   if (vec) { SGP_LAUNCH_UPDATE(4) } else { SGP_LAUNCH_UPDATE(1) }
 #undef SGP_LAUNCH_UPDATE
   SGP_RANK_TRY(r, cudaGetLastError());
   return SGP_OK;
+}
+
+int rank_overlap(sgp_rank *r, float *d_x, float *d_w, float *d_m, float *d_v, const float *d_g, float *d_z, int64_t k, int upd,
+                 const sgp::UpdateScalars &us, void *stream) {
+  if (r->tau < 1) return SGP_ERR_STATE;                  // without a delay the peers' messages are not there yet
+  int rc = check_device(r);
+  if (rc != SGP_OK) return rc;
+  sgp_rank_plan_t plan;
+  rc = sgp_rank_plan(r->sched, r->rank, k, r->tau, &plan);
+  if (rc != SGP_OK) return rc;
+  sgp::RankSources s;
+  rc = make_sources(r, plan, &s);
+  if (rc != SGP_OK) return rc;
+  sgp::RankParams p{};
+  fill_params(r, &p);
+  p.x = d_x;
+  p.w = d_w;
+  p.m = d_m;
+  p.v = d_v;
+  p.g = d_g;
+  p.z = d_z;
+  p.msg = r->block + static_cast<int64_t>(plan.write_slot) * r->slot_floats;
+  p.self_weight = plan.self_weight;
+  p.us = us;
+  const bool vec = aligned16(d_x) && aligned16(d_g) && (d_m == nullptr || aligned16(d_m)) && (d_v == nullptr || aligned16(d_v)) &&
+                   (d_z == nullptr || aligned16(d_z));
+  const unsigned grid = stream_grid(r, vec);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+#define SGP_LAUNCH_OVERLAP(VEC, HZ)                                                                                    \
+  switch (upd) {                                                                                                       \
+    case sgp::kUpdSgd: sgp::sgp_rank_overlap_kernel<VEC, sgp::kUpdSgd, HZ><<<grid, sgp::kRankThreads, 0, st>>>(p, s); break; \
+    case sgp::kUpdHeavyBall: sgp::sgp_rank_overlap_kernel<VEC, sgp::kUpdHeavyBall, HZ><<<grid, sgp::kRankThreads, 0, st>>>(p, s); break; \
+    case sgp::kUpdNesterov: sgp::sgp_rank_overlap_kernel<VEC, sgp::kUpdNesterov, HZ><<<grid, sgp::kRankThreads, 0, st>>>(p, s); break; \
+    default: sgp::sgp_rank_overlap_kernel<VEC, sgp::kUpdAdam, HZ><<<grid, sgp::kRankThreads, 0, st>>>(p, s);            \
+  }
+  if (vec) {
+    if (d_z) { SGP_LAUNCH_OVERLAP(4, true) } else { SGP_LAUNCH_OVERLAP(4, false) }
+  } else {
+    if (d_z) { SGP_LAUNCH_OVERLAP(1, true) } else { SGP_LAUNCH_OVERLAP(1, false) }
+  }
+#undef SGP_LAUNCH_OVERLAP
+  SGP_RANK_TRY(r, cudaGetLastError());
+  return SGP_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int sgp_rank_update(sgp_rank *r, const float *d_x, float *d_w, float *d_m, const float *d_g, int64_t k, float lr,
+                    float momentum, float weight_decay, int nesterov, void *stream) {
+  if (r == nullptr || d_x == nullptr || d_w == nullptr || d_g == nullptr || k < 0 || (momentum != 0.0f && d_m == nullptr))
+    return SGP_ERR_ARG;
+  return rank_update(r, d_x, d_w, momentum != 0.0f ? d_m : nullptr, nullptr, d_g, k, update_kind(momentum, nesterov),
+                     sgp::UpdateScalars{lr, momentum, weight_decay, 0.f, 0.f, 0.f, 0.f, 0.f}, stream);
+}
+
+int sgp_rank_update_adam(sgp_rank *r, const float *d_x, float *d_w, float *d_m1, float *d_m2, const float *d_g, int64_t k,
+                         int64_t t, float lr, float beta1, float beta2, float eps, float weight_decay, void *stream) {
+  if (r == nullptr || d_x == nullptr || d_w == nullptr || d_m1 == nullptr || d_m2 == nullptr || d_g == nullptr || k < 0 ||
+      !adam_args_ok(t, beta1, beta2, eps))
+    return SGP_ERR_ARG;
+  return rank_update(r, d_x, d_w, d_m1, d_m2, d_g, k, sgp::kUpdAdam, adam_scalars(lr, beta1, beta2, eps, weight_decay, t), stream);
 }
 
 int sgp_rank_mix(sgp_rank *r, float *d_x, float *d_w, float *d_z, int64_t k, void *stream) {
@@ -269,43 +348,18 @@ int sgp_rank_step_overlap(sgp_rank *r, float *d_x, float *d_w, float *d_m, const
                           float lr, float momentum, float weight_decay, int nesterov, void *stream) {
   if (r == nullptr || d_x == nullptr || d_w == nullptr || d_g == nullptr || k < 0 || (momentum != 0.0f && d_m == nullptr))
     return SGP_ERR_ARG;
-  if (r->tau < 1) return SGP_ERR_STATE;                  // without a delay the peers' messages are not there yet
-  int rc = check_device(r);
-  if (rc != SGP_OK) return rc;
-  sgp_rank_plan_t plan;
-  rc = sgp_rank_plan(r->sched, r->rank, k, r->tau, &plan);
-  if (rc != SGP_OK) return rc;
-  sgp::RankSources s;
-  rc = make_sources(r, plan, &s);
-  if (rc != SGP_OK) return rc;
-  sgp::RankParams p{};
-  fill_params(r, &p);
-  p.x = d_x;
-  p.w = d_w;
-  p.m = momentum != 0.0f ? d_m : nullptr;
-  p.g = d_g;
-  p.z = d_z;
-  p.msg = r->block + static_cast<int64_t>(plan.write_slot) * r->slot_floats;
-  p.self_weight = plan.self_weight;
-  p.us = sgp::UpdateScalars{lr, momentum, weight_decay, 0.f, 0.f, 0.f, 0.f, 0.f};
-  const bool vec = aligned16(d_x) && aligned16(d_g) && (p.m == nullptr || aligned16(p.m)) && (d_z == nullptr || aligned16(d_z));
-  const unsigned grid = stream_grid(r, vec);
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const int upd = update_kind(momentum, nesterov);
-#define SGP_LAUNCH_OVERLAP(VEC, HZ)                                                                                    \
-  switch (upd) {                                                                                                       \
-    case sgp::kUpdSgd: sgp::sgp_rank_overlap_kernel<VEC, sgp::kUpdSgd, HZ><<<grid, sgp::kRankThreads, 0, st>>>(p, s); break; \
-    case sgp::kUpdHeavyBall: sgp::sgp_rank_overlap_kernel<VEC, sgp::kUpdHeavyBall, HZ><<<grid, sgp::kRankThreads, 0, st>>>(p, s); break; \
-    default: sgp::sgp_rank_overlap_kernel<VEC, sgp::kUpdNesterov, HZ><<<grid, sgp::kRankThreads, 0, st>>>(p, s);        \
-  }
-  if (vec) {
-    if (d_z) { SGP_LAUNCH_OVERLAP(4, true) } else { SGP_LAUNCH_OVERLAP(4, false) }
-  } else {
-    if (d_z) { SGP_LAUNCH_OVERLAP(1, true) } else { SGP_LAUNCH_OVERLAP(1, false) }
-  }
-#undef SGP_LAUNCH_OVERLAP
-  SGP_RANK_TRY(r, cudaGetLastError());
-  return SGP_OK;
+  return rank_overlap(r, d_x, d_w, momentum != 0.0f ? d_m : nullptr, nullptr, d_g, d_z, k, update_kind(momentum, nesterov),
+                      sgp::UpdateScalars{lr, momentum, weight_decay, 0.f, 0.f, 0.f, 0.f, 0.f}, stream);
+}
+
+int sgp_rank_step_overlap_adam(sgp_rank *r, float *d_x, float *d_w, float *d_m1, float *d_m2, const float *d_g, float *d_z,
+                               int64_t k, int64_t t, float lr, float beta1, float beta2, float eps, float weight_decay,
+                               void *stream) {
+  if (r == nullptr || d_x == nullptr || d_w == nullptr || d_m1 == nullptr || d_m2 == nullptr || d_g == nullptr || k < 0 ||
+      !adam_args_ok(t, beta1, beta2, eps))
+    return SGP_ERR_ARG;
+  return rank_overlap(r, d_x, d_w, d_m1, d_m2, d_g, d_z, k, sgp::kUpdAdam, adam_scalars(lr, beta1, beta2, eps, weight_decay, t),
+                      stream);
 }
 
 int sgp_rank_device_status(sgp_rank *r, unsigned *status) {

@@ -64,6 +64,20 @@ class LoopbackGroup:
                 rk.step_overlap(xs[r], ws[r], m_of(r), gs[r], z_of(r), k, lr, momentum, weight_decay, nesterov,
                                 stream=stream)
 
+    def step_adam(self, xs, ws, m1s, m2s, gs, zs, k: int, t: int, lr: float, beta1: float = 0.9, beta2: float = 0.999,
+                  eps: float = 1e-8, weight_decay: float = 0.0, stream=None) -> None:
+        """The same protocol with the Adam preconditioner (m1s[r], m2s[r]: rank r's moment rows)."""
+        z_of = (lambda r: zs[r]) if zs is not None else (lambda r: None)
+        if self.tau == 0:
+            for r, rk in enumerate(self.ranks):
+                rk.update_adam(xs[r], ws[r], m1s[r], m2s[r], gs[r], k, t, lr, beta1, beta2, eps, weight_decay, stream=stream)
+            for r, rk in enumerate(self.ranks):
+                rk.mix(xs[r], ws[r], z_of(r), k, stream=stream)
+        else:
+            for r, rk in enumerate(self.ranks):
+                rk.step_overlap_adam(xs[r], ws[r], m1s[r], m2s[r], gs[r], z_of(r), k, t, lr, beta1, beta2, eps,
+                                     weight_decay, stream=stream)
+
     def device_status(self) -> int:
         status = 0
         for rk in self.ranks:
@@ -129,5 +143,17 @@ class DistributedRank:
                 self.node.mix(x, w, z, k)
             elif call == "step_overlap":
                 self.node.step_overlap(x, w, m if momentum != 0.0 else None, g, z, k, lr, momentum, weight_decay, nesterov)
+            else:
+                self.barrier()
+
+    def step_adam(self, x, w, m1, m2, g, z, k: int, t: int, lr: float, beta1: float = 0.9, beta2: float = 0.999,
+                  eps: float = 1e-8, weight_decay: float = 0.0) -> None:
+        for call in step_protocol(self.tau):
+            if call == "update":
+                self.node.update_adam(x, w, m1, m2, g, k, t, lr, beta1, beta2, eps, weight_decay)
+            elif call == "mix":
+                self.node.mix(x, w, z, k)
+            elif call == "step_overlap":
+                self.node.step_overlap_adam(x, w, m1, m2, g, z, k, t, lr, beta1, beta2, eps, weight_decay)
             else:
                 self.barrier()

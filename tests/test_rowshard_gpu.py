@@ -223,3 +223,42 @@ def test_two_processes_share_slots_through_cuda_ipc(binding, inputs, tau):
         assert_close(f"z[{r}]", z, st.z[r])
         assert_close(f"m[{r}]", m, st.u[r])
         assert abs(wt - st.w[r]) <= 1e-6
+
+
+@pytest.mark.parametrize("n,d,tau,graph", [(8, 4_100, 0, "exp"), (8, 4_101, 1, "exp"), (16, 3_000, 2, "random")])
+def test_loopback_adam_matches_oracle_and_stacked_step(binding, inputs, n, d, tau, graph):
+    """Adam-SGP one node per GPU (Sec. 6.2: the paper's 8-node Transformer runs): moments stay on the node, the mix is
+    the same; bit-identical to sgp_step_adam on the stacked arrays."""
+    from oracle import sgp as osgp
+    from paper_1811_10792_b200 import rowshard
+    w = dataclasses.replace(inputs.sweep_workload(n, d), graph=graph, peers=2, tau=tau, optimizer="adam", lr=1e-2)
+    K, b1, b2, eps, wd = 6, 0.9, 0.98, 1e-8, 1e-3
+    X = inputs.initial_x(w, device=DEV).contiguous()
+    x0 = X.cpu().numpy().astype(np.float64)
+    W = torch.ones(n, device=DEV); M1 = torch.zeros_like(X); M2 = torch.zeros_like(X); Z = torch.empty_like(X)
+    G = torch.empty_like(X)
+    xs = [X[r].clone() for r in range(n)]
+    m1s = [torch.zeros(d, device=DEV) for _ in range(n)]
+    m2s = [torch.zeros(d, device=DEV) for _ in range(n)]
+    zs = [torch.empty(d, device=DEV) for _ in range(n)]
+    ws = [torch.ones(1, device=DEV) for _ in range(n)]
+    grads = []
+    with binding.Sgp(n, d, graph_desc(w, binding), tau=tau) as h, \
+            rowshard.LoopbackGroup(n, d, graph_desc(w, binding), tau=tau) as grp:
+        for k in range(K):
+            inputs.gradient(w, k, G)
+            grads.append(G.cpu().numpy().astype(np.float64))
+            gs = [G[r].clone() for r in range(n)]
+            grp.step_adam(xs, ws, m1s, m2s, gs, zs, k, k + 1, w.lr, b1, b2, eps, wd)
+            h.step_adam(X, W, M1, M2, G, Z, k, k + 1, w.lr, b1, b2, eps, wd)
+        torch.cuda.synchronize()
+        assert grp.device_status() == 0
+    st = osgp.sgp_run(x0, K, oracle_P_of_k(w), lambda k, z: grads[k], w.lr, weight_decay=wd, tau=tau, adam=(b1, b2, eps))
+    got = dict(X=torch.stack(xs), Z=torch.stack(zs), M1=torch.stack(m1s), M2=torch.stack(m2s), W=torch.cat(ws))
+    assert_close("X", got["X"].cpu().numpy(), st.x)
+    assert_close("Z", got["Z"].cpu().numpy(), st.z)
+    assert_close("M1", got["M1"].cpu().numpy(), st.u)
+    assert_close("M2", got["M2"].cpu().numpy(), st.v)
+    assert_close("W", got["W"].cpu().numpy(), st.w)
+    for name, ref in (("X", X), ("Z", Z), ("M1", M1), ("M2", M2), ("W", W)):
+        assert torch.equal(got[name], ref), name
