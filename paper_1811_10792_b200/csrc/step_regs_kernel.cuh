@@ -80,13 +80,26 @@ sgp_step_regs_kernel(const __grid_constant__ StepParams p, const __grid_constant
           if (DIAG && HAS_RING) rr[q] = diag_ring_sum<V>(p, off[q], nullptr);
         }
       }
+      if constexpr (kGatherFirst) {
+        // the same ordering in this phase: every update of the batch, then every momentum store (another +0.3 to
+        // +0.5 %); x[q] becomes the half step
+#pragma unroll
+        for (int q = 0; q < kItemsPerThread; ++q)
+          if (ok[q]) x[q] = local_update<UPD, V>(x[q], g[q], u[q], vv[q], p);
+#pragma unroll
+        for (int q = 0; q < kItemsPerThread; ++q)
+          if (ok[q]) st_stream(reinterpret_cast<V *>(p.M + off[q]), u[q]);
+      }
 #pragma unroll
       for (int q = 0; q < kItemsPerThread; ++q) {
         const int item = base + q * kThreads + threadIdx.x;
         if (ok[q]) {
-          const V h = local_update<UPD, V>(x[q], g[q], u[q], vv[q], p);
-          if (HAS_M) st_stream(reinterpret_cast<V *>(p.M + off[q]), u[q]);
-          if (HAS_V) st_stream(reinterpret_cast<V *>(p.V + off[q]), vv[q]);
+          V h = x[q];
+          if constexpr (!kGatherFirst) {
+            h = local_update<UPD, V>(x[q], g[q], u[q], vv[q], p);
+            if (HAS_M) st_stream(reinterpret_cast<V *>(p.M + off[q]), u[q]);
+            if (HAS_V) st_stream(reinterpret_cast<V *>(p.V + off[q]), vv[q]);
+          }
           H[item] = h;
           if (DIAG) {
             csum = vadd(csum, h);
