@@ -45,7 +45,8 @@ def build(force: bool = False, verbose: bool = False, extra_flags=(), lib_path: 
         return lib_path
     from concurrent.futures import ThreadPoolExecutor
     tag = os.path.splitext(os.path.basename(lib_path))[0]
-    obj_dir = os.path.join(PKG_DIR, "build", tag)
+    import tempfile
+    obj_dir = os.path.join(tempfile.gettempdir(), "sgp_build_%d" % os.getuid(), tag)      # objects stay out of the tree
     os.makedirs(obj_dir, exist_ok=True)
     inc = ["-I", os.path.join(ROOT, "include"), "-I", CSRC]
 
