@@ -43,10 +43,18 @@ inline int update_kind(float momentum, int nesterov) {
   return nesterov != 0 ? sgp::kUpdNesterov : sgp::kUpdHeavyBall;
 }
 
-unsigned stream_grid(const sgp_rank *r, bool vec) {
+// Grid of a streaming rank kernel: exactly the CTAs that are resident at once (one wave, grid-stride inside), so
+// that no partial second wave is left at the end of a launch that lasts only ~100 us.
+template <typename Kernel>
+unsigned stream_grid(const sgp_rank *r, bool vec, Kernel kern) {
   const int64_t work = vec ? std::max<int64_t>(1, r->d >> 2) : r->d;
+  int per_sm = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, sgp::kRankThreads, 0) != cudaSuccess || per_sm < 1) {
+    (void)cudaGetLastError();
+    per_sm = 4;
+  }
   return static_cast<unsigned>(std::max<int64_t>(1, std::min<int64_t>((work + sgp::kRankThreads - 1) / sgp::kRankThreads,
-                                                                      static_cast<int64_t>(r->sm_count) * 8)));
+                                                                      static_cast<int64_t>(r->sm_count) * per_sm)));
 }
 
 int check_device(const sgp_rank *r) {
@@ -236,14 +244,14 @@ int rank_update(sgp_rank *r, const float *d_x, float *d_w, float *d_m, float *d_
   p.msg = r->block + (k % r->slots) * r->slot_floats;
   p.us = us;
   const bool vec = aligned16(d_x) && aligned16(d_g) && (d_m == nullptr || aligned16(d_m)) && (d_v == nullptr || aligned16(d_v));
-  const unsigned grid = stream_grid(r, vec);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-#define SGP_LAUNCH_UPDATE(VEC)                                                                                   \
-  switch (upd) {                                                                                                 \
-    case sgp::kUpdSgd: sgp::sgp_rank_update_kernel<VEC, sgp::kUpdSgd><<<grid, sgp::kRankThreads, 0, st>>>(p); break; \
-    case sgp::kUpdHeavyBall: sgp::sgp_rank_update_kernel<VEC, sgp::kUpdHeavyBall><<<grid, sgp::kRankThreads, 0, st>>>(p); break; \
-    case sgp::kUpdNesterov: sgp::sgp_rank_update_kernel<VEC, sgp::kUpdNesterov><<<grid, sgp::kRankThreads, 0, st>>>(p); break; \
-    default: sgp::sgp_rank_update_kernel<VEC, sgp::kUpdAdam><<<grid, sgp::kRankThreads, 0, st>>>(p);              \
+#define SGP_LAUNCH_ONE(KERNEL, ...) KERNEL<<<stream_grid(r, vec, KERNEL), sgp::kRankThreads, 0, st>>>(__VA_ARGS__)
+#define SGP_LAUNCH_UPDATE(VEC)                                                                  \
+  switch (upd) {                                                                                \
+    case sgp::kUpdSgd: SGP_LAUNCH_ONE((sgp::sgp_rank_update_kernel<VEC, sgp::kUpdSgd>), p); break; \
+    case sgp::kUpdHeavyBall: SGP_LAUNCH_ONE((sgp::sgp_rank_update_kernel<VEC, sgp::kUpdHeavyBall>), p); break; \
+    case sgp::kUpdNesterov: SGP_LAUNCH_ONE((sgp::sgp_rank_update_kernel<VEC, sgp::kUpdNesterov>), p); break; \
+    default: SGP_LAUNCH_ONE((sgp::sgp_rank_update_kernel<VEC, sgp::kUpdAdam>), p);               \
   }
   if (vec) { SGP_LAUNCH_UPDATE(4) } else { SGP_LAUNCH_UPDATE(1) }
 #undef SGP_LAUNCH_UPDATE
@@ -275,14 +283,13 @@ int rank_overlap(sgp_rank *r, float *d_x, float *d_w, float *d_m, float *d_v, co
   p.us = us;
   const bool vec = aligned16(d_x) && aligned16(d_g) && (d_m == nullptr || aligned16(d_m)) && (d_v == nullptr || aligned16(d_v)) &&
                    (d_z == nullptr || aligned16(d_z));
-  const unsigned grid = stream_grid(r, vec);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-#define SGP_LAUNCH_OVERLAP(VEC, HZ)                                                                                    \
-  switch (upd) {                                                                                                       \
-    case sgp::kUpdSgd: sgp::sgp_rank_overlap_kernel<VEC, sgp::kUpdSgd, HZ><<<grid, sgp::kRankThreads, 0, st>>>(p, s); break; \
-    case sgp::kUpdHeavyBall: sgp::sgp_rank_overlap_kernel<VEC, sgp::kUpdHeavyBall, HZ><<<grid, sgp::kRankThreads, 0, st>>>(p, s); break; \
-    case sgp::kUpdNesterov: sgp::sgp_rank_overlap_kernel<VEC, sgp::kUpdNesterov, HZ><<<grid, sgp::kRankThreads, 0, st>>>(p, s); break; \
-    default: sgp::sgp_rank_overlap_kernel<VEC, sgp::kUpdAdam, HZ><<<grid, sgp::kRankThreads, 0, st>>>(p, s);            \
+#define SGP_LAUNCH_OVERLAP(VEC, HZ)                                                                          \
+  switch (upd) {                                                                                             \
+    case sgp::kUpdSgd: SGP_LAUNCH_ONE((sgp::sgp_rank_overlap_kernel<VEC, sgp::kUpdSgd, HZ>), p, s); break;    \
+    case sgp::kUpdHeavyBall: SGP_LAUNCH_ONE((sgp::sgp_rank_overlap_kernel<VEC, sgp::kUpdHeavyBall, HZ>), p, s); break; \
+    case sgp::kUpdNesterov: SGP_LAUNCH_ONE((sgp::sgp_rank_overlap_kernel<VEC, sgp::kUpdNesterov, HZ>), p, s); break; \
+    default: SGP_LAUNCH_ONE((sgp::sgp_rank_overlap_kernel<VEC, sgp::kUpdAdam, HZ>), p, s);                    \
   }
   if (vec) {
     if (d_z) { SGP_LAUNCH_OVERLAP(4, true) } else { SGP_LAUNCH_OVERLAP(4, false) }
@@ -331,14 +338,13 @@ int sgp_rank_mix(sgp_rank *r, float *d_x, float *d_w, float *d_z, int64_t k, voi
   p.w = d_w;
   p.z = d_z;
   const bool vec = aligned16(d_x) && (d_z == nullptr || aligned16(d_z));
-  const unsigned grid = stream_grid(r, vec);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (vec) {
-    if (d_z) sgp::sgp_rank_mix_kernel<4, true><<<grid, sgp::kRankThreads, 0, st>>>(p, s);
-    else sgp::sgp_rank_mix_kernel<4, false><<<grid, sgp::kRankThreads, 0, st>>>(p, s);
+    if (d_z) SGP_LAUNCH_ONE((sgp::sgp_rank_mix_kernel<4, true>), p, s);
+    else SGP_LAUNCH_ONE((sgp::sgp_rank_mix_kernel<4, false>), p, s);
   } else {
-    if (d_z) sgp::sgp_rank_mix_kernel<1, true><<<grid, sgp::kRankThreads, 0, st>>>(p, s);
-    else sgp::sgp_rank_mix_kernel<1, false><<<grid, sgp::kRankThreads, 0, st>>>(p, s);
+    if (d_z) SGP_LAUNCH_ONE((sgp::sgp_rank_mix_kernel<1, true>), p, s);
+    else SGP_LAUNCH_ONE((sgp::sgp_rank_mix_kernel<1, false>), p, s);
   }
   SGP_RANK_TRY(r, cudaGetLastError());
   return SGP_OK;
