@@ -276,6 +276,11 @@ int sgp_param_deviation(sgp_handle *h, const float *d_A, double *h_dev, void *st
  *   "stages"       shared-memory stages of the bulk-copy pipeline (0 = automatic, at most 8)
  *   "single_buffer" register-staged kernel: 0 = automatic (n > 128), 1 = one exchange tile and two barriers
  *                  per tile, 2 = two exchange tiles and one barrier
+ *   "lockstep"     register-staged kernel: 2 or 4 = launch it as thread-block clusters of that many CTAs that take
+ *                  neighbouring tiles and meet at a cluster barrier before each tile (they share no data; it only
+ *                  aligns their memory traffic in time), 1 = independent CTAs, 0 = automatic (clusters when rows do
+ *                  not start on 128-byte boundaries, where they win back about 4 % of the bandwidth, and for
+ *                  tau >= 1 at 1 KB row segments).  Results do not depend on it, bit for bit.
  *   "wait_limit_ms" bound of every in-kernel wait of the pipelined kernel (0 = 2000 ms); a wait that runs out
  *                  sets the device status word (sgp_device_status) and the CTA leaves: nothing hangs
  *   "inject_stall" test hook, 0/1: one CTA of the pipelined kernel never requests its first tile, so that
@@ -291,7 +296,7 @@ int sgp_param_deviation(sgp_handle *h, const float *d_A, double *h_dev, void *st
  *                  (sum_i x_i' plus ring against sum_i h_i plus ring, Sec. 2); a drift sets SGP_STATUS_COLUMN_SUM in
  *                  the device status word.  Costs about two extra passes over the arrays and 8 d bytes of device
  *                  memory, allocated when the option is switched on (SGP_ERR_ALLOC if that fails)
- * Read-only through sgp_get_option: "last_variant", "last_grid", "last_smem", "last_tile_cols" describe
+ * Read-only through sgp_get_option: "last_variant", "last_grid", "last_smem", "last_tile_cols", "last_lockstep" describe
  * the most recent step launch of the handle (which kernel ran, CTAs, dynamic shared memory, tile width);
  * "launches" counts the step kernels the handle has launched so far.
  * Unknown keys or unsupported values return SGP_ERR_ARG and change nothing.

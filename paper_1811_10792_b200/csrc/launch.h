@@ -24,6 +24,7 @@ struct LaunchRecord {
   int64_t grid = 0;
   int64_t smem = 0;
   int64_t tile_cols = 0;
+  int lockstep = 0;      // CTAs per lockstep cluster of the register-staged kernel (0 = independent CTAs)
   int cuda_error = 0;
 };
 
@@ -37,6 +38,9 @@ struct KernelInfo {
   size_t enabled_smem = 48 * 1024;
 };
 int kernel_info(int device, const void *kern, size_t smem, KernelInfo *out, int *cuda_error);
+// Clusters of `cluster` CTAs (kThreads threads, `smem` dynamic bytes each) of `kern` that `device` holds at once;
+// 0 when the query fails.  Cached per (device, kernel, cluster, smem).
+int resident_clusters(int device, const void *kern, int cluster, size_t smem);
 
 // Register-staged kernel: one exchange tile (two barriers per tile) where that keeps the row segments long.
 bool auto_single_buffer(int n);
@@ -50,6 +54,7 @@ struct RegsOptions {
   bool tile_cols_forced = false;  // true: the caller asked for exactly this width (no narrowing for short rows)
   int cps = 0;                    // CTAs per SM, 0 = as many as are resident
   int single_buffer = 0;          // 0 automatic, 1 one tile, 2 two tiles
+  int lockstep = 0;               // 0 automatic, 1 independent CTAs, 2 / 4 = clusters of that many CTAs in lockstep
 };
 
 // One launch of the register-staged kernel over columns [p.col_begin, p.col_end) with vector width vec (4 or 1).

@@ -2,6 +2,7 @@
 #include <algorithm>
 #include <map>
 #include <mutex>
+#include <tuple>
 #include <utility>
 
 #include "launch.h"
@@ -59,6 +60,32 @@ int kernel_info(int device, const void *kern, size_t smem, KernelInfo *out, int 
   }
   *out = it->second;
   return SGP_OK;
+}
+
+int resident_clusters(int device, const void *kern, int cluster, size_t smem) {
+  static std::map<std::tuple<int, const void *, int, size_t>, int> cache;
+  std::lock_guard<std::mutex> lock(g_kernel_info_mutex);
+  const auto key = std::make_tuple(device, kern, cluster, smem);
+  auto it = cache.find(key);
+  if (it != cache.end()) return it->second;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(static_cast<unsigned>(cluster));
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cudaLaunchAttribute attr{};
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = static_cast<unsigned>(cluster);
+  attr.val.clusterDim.y = 1;
+  attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  int clusters = 0;
+  if (cudaOccupancyMaxActiveClusters(&clusters, kern, &cfg) != cudaSuccess) {
+    (void)cudaGetLastError();
+    clusters = 0;
+  }
+  cache.emplace(key, clusters);
+  return clusters;
 }
 
 // One exchange tile (two barriers per tile) where that keeps the row segments long (n = 64: 1 KB segments 0.95
@@ -134,10 +161,48 @@ int launch_regs(const DeviceInfo &dev, StepParams p, const ConstTable *ct, int u
     const int by_smem = static_cast<int>((227 * 1024) / (smem + ki.static_smem + 1024));
     cps = std::max(1, std::min({by_regs, by_smem, 2048 / kThreads}));
   }
-  const int64_t grid = std::min<int64_t>(ntiles, static_cast<int64_t>(dev.sm_count) * cps);
+  int64_t grid = std::min<int64_t>(ntiles, static_cast<int64_t>(dev.sm_count) * cps);
   static const ConstTable kEmptyTable{};
-  kern<<<static_cast<unsigned>(grid), kThreads, smem, stream>>>(p, ct != nullptr ? *ct : kEmptyTable);
-  const cudaError_t e = cudaGetLastError();
+  // Lockstep clusters (what was measured, of the copy bandwidth): rows that do not start on 128-byte boundaries
+  // split every 1 KB block between two tiles, and CTAs that take neighbouring tiles at the same moment get most of
+  // the loss back (rows on 32-byte boundaries, n = 32: 0.87 -> 0.91 in pairs; tau = 1: 0.86 -> 0.90; n = 64:
+  // 0.83 -> 0.88 in pairs, 0.91 in fours; n = 128: 0.61 -> 0.66 / 0.74); a cluster of four leaves 12 of the 296 CTA
+  // slots empty, which costs n = 32 more than it returns (0.89).  With rows on 1 KB boundaries pairs are worth
+  // +0.6 % with a delay ring at 1 KB segments and -1 to -3 % with narrow (n >= 96) or wide (n <= 24) tiles: off.
+  p.lockstep = 0;
+  if (opt.lockstep >= 2) {
+    p.lockstep = opt.lockstep;
+  } else if (opt.lockstep == 0 && vec == 4 && n >= 32 && ntiles >= 2 * grid) {
+    const uintptr_t bits = reinterpret_cast<uintptr_t>(p.X) | reinterpret_cast<uintptr_t>(p.G) | reinterpret_cast<uintptr_t>(p.M) |
+                           reinterpret_cast<uintptr_t>(p.V) | reinterpret_cast<uintptr_t>(p.Z) | reinterpret_cast<uintptr_t>(p.ring_x) |
+                           static_cast<uintptr_t>(p.ld * 4);
+    if ((bits & 127) != 0 && tile_cols <= 256) p.lockstep = n >= 64 ? 4 : 2;
+    else if ((bits & 1023) == 0 && has_ring && tile_cols == 256) p.lockstep = 2;
+  }
+  cudaError_t e = cudaSuccess;
+  if (p.lockstep) {
+    const int clusters = resident_clusters(dev.device, reinterpret_cast<const void *>(kern), p.lockstep, smem);
+    if (clusters < 1) p.lockstep = 0;
+    else grid = std::min<int64_t>({(ntiles + p.lockstep - 1) / p.lockstep, static_cast<int64_t>(clusters), static_cast<int64_t>(dev.sm_count) * cps / p.lockstep}) * p.lockstep;
+  }
+  if (p.lockstep) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(static_cast<unsigned>(grid));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = static_cast<unsigned>(p.lockstep);
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, kern, p, ct != nullptr ? *ct : kEmptyTable);
+  } else {
+    kern<<<static_cast<unsigned>(grid), kThreads, smem, stream>>>(p, ct != nullptr ? *ct : kEmptyTable);
+    e = cudaGetLastError();
+  }
   if (e != cudaSuccess) {
     rec->cuda_error = static_cast<int>(e);
     return SGP_ERR_CUDA;
@@ -146,6 +211,7 @@ int launch_regs(const DeviceInfo &dev, StepParams p, const ConstTable *ct, int u
   rec->grid = grid;
   rec->smem = static_cast<int64_t>(smem);
   rec->tile_cols = tile_cols;
+  rec->lockstep = p.lockstep;
   return SGP_OK;
 }
 

@@ -48,7 +48,7 @@ struct sgp_handle {
   double *d_stats = nullptr;    // kDevStatsCount doubles
   double *d_expect = nullptr;   // d doubles, allocated when "check_steps" is switched on
   int64_t opt_variant = 0, opt_tile_cols = 0, opt_ctas_per_sm = 0, opt_stages = 0, opt_l2_hint = 0, opt_single_buffer = 0, opt_wait_limit_ms = 0,
-          opt_inject_stall = 0, opt_send_period = 1, opt_diagnostics = 0, opt_check_steps = 0, opt_cluster = 0;
+          opt_inject_stall = 0, opt_send_period = 1, opt_diagnostics = 0, opt_check_steps = 0, opt_cluster = 0, opt_lockstep = 0;
   sgp::LaunchRecord last;       // of the most recent step launch
   int64_t launches = 0;         // step kernels launched so far
   bool diag_valid = false;      // a step with diagnostics has been enqueued since the last reset
@@ -259,6 +259,7 @@ int launch_regs(sgp_handle *h, const StepArgs &a, const Plan &pl, int64_t c0, in
   opt.tile_cols_forced = h->opt_tile_cols > 0;
   opt.cps = pl.cps;
   opt.single_buffer = static_cast<int>(h->opt_single_buffer);
+  opt.lockstep = static_cast<int>(h->opt_lockstep);
   sgp::LaunchRecord rec;
   const int rc = sgp::launch_regs(h->dev, p, h->const_ok[slot] ? &h->const_tables[slot] : nullptr, a.upd, vec,
                                   csr_of(h, slot).uniform_rows, opt, stream, &rec);
@@ -343,6 +344,12 @@ int launch_step_range(sgp_handle *h, const StepArgs &a, int64_t c0, int64_t c1, 
     Plan pl = make_plan(h, arrays, a.M != nullptr, nnz, true);
     // short rows (fewer 1 KB tiles than SMs): the register kernel with narrow tiles spreads them better
     if (h->opt_variant == 0 && pl.variant >= 2 && (vec_end - c0) < int64_t{256} * h->dev.sm_count) pl = Plan{1, 256, 2, 0};
+    // rows that do not start on 128-byte boundaries (a dense pitch): the register-staged kernel in lockstep pairs
+    // reaches 0.91 of the copy bandwidth at n = 32 where the pipelined kernel reaches 0.89
+    const uintptr_t row_bits = reinterpret_cast<uintptr_t>(a.X) | reinterpret_cast<uintptr_t>(a.G) | reinterpret_cast<uintptr_t>(a.M) |
+                               reinterpret_cast<uintptr_t>(a.Z) | static_cast<uintptr_t>(h->ld * 4);
+    if (h->opt_variant == 0 && h->opt_lockstep != 1 && pl.variant >= 2 && a.M != nullptr && (row_bits & 127) != 0)
+      pl = Plan{1, sgp::regs_tile_cols(h->n, 4 * 1024), 2, 0};
     int rc = SGP_ERR_STATE;
     // Opt-in (variant 4): a cluster of CTAs shares the tile through distributed shared memory, so that row segments
     // stay 1 KB long at n = 256 (256 bytes with one CTA).  Measured slower than the one-CTA kernel at every shape
@@ -909,6 +916,9 @@ int sgp_set_option(sgp_handle *h, const char *key, int64_t value) {
   } else if (std::strcmp(key, "single_buffer") == 0) {
     if (value > 2) return SGP_ERR_ARG;
     h->opt_single_buffer = value;
+  } else if (std::strcmp(key, "lockstep") == 0) {
+    if (value != 0 && value != 1 && value != 2 && value != 4) return SGP_ERR_ARG;
+    h->opt_lockstep = value;
   } else if (std::strcmp(key, "l2_hint") == 0) {
     if (value > 4) return SGP_ERR_ARG;
     h->opt_l2_hint = value;
@@ -954,6 +964,7 @@ int sgp_get_option(const sgp_handle *h, const char *key, int64_t *value) {
   else if (std::strcmp(key, "stages") == 0) *value = h->opt_stages;
   else if (std::strcmp(key, "l2_hint") == 0) *value = h->opt_l2_hint;
   else if (std::strcmp(key, "single_buffer") == 0) *value = h->opt_single_buffer;
+  else if (std::strcmp(key, "lockstep") == 0) *value = h->opt_lockstep;
   else if (std::strcmp(key, "wait_limit_ms") == 0) *value = h->opt_wait_limit_ms;
   else if (std::strcmp(key, "inject_stall") == 0) *value = h->opt_inject_stall;
   else if (std::strcmp(key, "send_period") == 0) *value = h->opt_send_period;
@@ -965,6 +976,7 @@ int sgp_get_option(const sgp_handle *h, const char *key, int64_t *value) {
   else if (std::strcmp(key, "launches") == 0) *value = h->launches;
   else if (std::strcmp(key, "last_smem") == 0) *value = h->last.smem;
   else if (std::strcmp(key, "last_tile_cols") == 0) *value = h->last.tile_cols;
+  else if (std::strcmp(key, "last_lockstep") == 0) *value = h->last.lockstep;
   else return SGP_ERR_ARG;
   return SGP_OK;
 }

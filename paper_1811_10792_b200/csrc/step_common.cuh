@@ -69,6 +69,8 @@ struct StepParams {
   int inject_stall;    // TMA kernel, fault-injection for tests: CTA 0 never requests its first tile, so its
                        // consumers' bounded wait runs out and the status word is set (nothing hangs)
   int biased;          // 1: z = x, the push-sum weight is left out of the de-bias (Table 4, biased OSGP)
+  int lockstep;        // register kernel: > 0 = launched as clusters of this many CTAs that take neighbouring tiles and
+                       // meet at a cluster barrier before each tile (no data is shared between them)
   float lr, momentum, wd;
   // Adam only: decay rates, epsilon, lr / (1 - beta1^t) and 1 / sqrt(1 - beta2^t)
   float beta1, beta2, eps, adam_step, adam_rsqrt_bc2;

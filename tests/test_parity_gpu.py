@@ -474,6 +474,42 @@ def test_cluster_kernel_matches_oracle_and_register_kernel(binding, inputs, n, d
         assert np.array_equal(a[name], b[name]), name
 
 
+# ------------------------------------------------------------------ lockstep clusters of the register-staged kernel
+@pytest.mark.parametrize("n,d,tau,size,diag", [(32, 1_029, 0, 2, 0), (32, 70_001, 1, 2, 0), (64, 9_003, 0, 4, 0), (5, 2_000, 2, 4, 0),
+                                               (130, 2_052, 0, 4, 0), (2, 260, 0, 2, 0), (48, 40_000, 1, 2, 1), (8, 300_001, 0, 4, 1)])
+def test_lockstep_clusters_change_no_bit(binding, inputs, n, d, tau, size, diag):
+    """CTAs launched as clusters that meet before each tile share no data: the step's results are those of independent
+    CTAs bit for bit and within tolerance of the oracle.  The shapes leave the last cluster with fewer tiles than CTAs
+    (1,029 columns are 5 tiles of 256), use the delay ring, the scalar tail and the fused diagnostics."""
+    w = dataclasses.replace(inputs.sweep_workload(n, d), tau=tau, weight_decay=1e-3, K=5)
+    a = _run_gpu(binding, inputs, w, options={"variant": 1, "lockstep": size, "diagnostics": diag})
+    _compare(w, a)
+    b = _run_gpu(binding, inputs, w, options={"variant": 1, "lockstep": 1, "diagnostics": diag})
+    for name in ("X", "Z", "M", "W"):
+        assert np.array_equal(a[name], b[name]), name
+
+
+def test_lockstep_is_automatic_for_rows_off_the_128_byte_grid(binding, inputs):
+    """A dense pitch whose rows start on 32-byte boundaries takes the register-staged kernel in lockstep pairs; the same
+    step with rows on 1 KB boundaries does not; both give the same bits."""
+    w = dataclasses.replace(inputs.sweep_workload(32, 400_008), K=1)
+    assert (w.d * 4) % 128 == 32
+    results = []
+    for ld in (w.d, (w.d + 255) // 256 * 256):
+        X = inputs.initial_x(w, device=DEV, ld=ld)
+        M = torch.zeros((w.n, ld), device=DEV)[:, :w.d]; Z = torch.empty((w.n, ld), device=DEV)[:, :w.d]
+        G = inputs.gradient(w, 0, torch.empty((w.n, ld), device=DEV)[:, :w.d])
+        W = torch.ones(w.n, device=DEV)
+        with binding.Sgp(w.n, w.d, graph_desc(w, binding), ld=ld) as h:
+            h.step(X, W, M, G, Z, 0, w.lr, w.momentum, 0.0, True)
+            torch.cuda.synchronize()
+            assert h.device_status() == 0
+            results.append((h.get_option("last_lockstep"), h.get_option("last_variant"), h.get_option("last_grid"), Z.cpu().numpy().copy()))
+    assert results[0][0] == 2 and results[0][1] == 1 and results[0][2] % 2 == 0
+    assert results[1][0] == 0
+    assert np.array_equal(results[0][3], results[1][3])
+
+
 def test_cluster_kernel_is_opt_in(binding, inputs):
     w = inputs.sweep_workload(256, 300_000)
     X = inputs.initial_x(w, device=DEV).contiguous()
