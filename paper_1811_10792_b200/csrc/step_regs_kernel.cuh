@@ -51,13 +51,16 @@ sgp_step_regs_kernel(const __grid_constant__ StepParams p, const __grid_constant
 
   // Lockstep clusters: the CTAs of a cluster take neighbouring tiles and start each tile together, so that the parts
   // of a 1 KB block of a row that straddles their common tile edge are requested at about the same time.  Nothing
-  // is shared between them; the barrier only aligns them in time.
-  unsigned pair_rank = 0;
-  if (p.lockstep) asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(pair_rank));
-  for (int64_t tile0 = static_cast<int64_t>(blockIdx.x) - pair_rank; tile0 < ntiles; tile0 += gridDim.x) {
-    const int64_t tile = tile0 + pair_rank;
-    if (p.lockstep) asm volatile("barrier.cluster.arrive.relaxed.aligned;\n\tbarrier.cluster.wait.aligned;" ::: "memory");
-    if (tile >= ntiles) continue;            // the odd CTA past the last tile only keeps the barrier count
+  // is shared between them; the barrier only aligns them in time.  (Written so that nothing but `tile` lives across
+  // the loop: the instantiations at the register cap lose 1 % to one more live value.)
+  for (int64_t tile = blockIdx.x;; tile += gridDim.x) {
+    if (p.lockstep) {
+      unsigned rank_in_cluster;
+      asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank_in_cluster));
+      if (tile - rank_in_cluster >= ntiles) break;      // the whole cluster is past the last tile
+      asm volatile("barrier.cluster.arrive.relaxed.aligned;\n\tbarrier.cluster.wait.aligned;" ::: "memory");
+    }
+    if (tile >= ntiles) break;                           // a CTA past the last tile has kept the barrier count
     const int64_t col0 = p.col_begin + tile * tile_cols;
     V *H = buf ? H1 : H0;
     V csum = vzero<V>(), rsum = vzero<V>();      // diagnostics: this thread's share of its column's sums
