@@ -192,7 +192,8 @@ int sgp_debias(sgp_handle *h, const float *d_X, const float *d_W, float *d_Z, vo
  * device->host copy overlap with the neighbouring chunks on the handle's three internal streams.
  * Work the caller already enqueued on `stream` is waited for on the device (an event, no host
  * synchronisation on entry).  Returns after everything has completed (synchronises the internal streams).
- * chunk_cols <= 0 picks a default.
+ * chunk_cols <= 0 picks a default (about 64 MB of gradient per chunk, with smaller chunks at both ends so that
+ * the pipeline fills and drains quickly); a positive value cuts the columns into equal chunks of that width.
  */
 int sgp_step_host(sgp_handle *h, float *d_X, float *d_W, float *d_M, const float *h_G, float *h_Z,
                   float *d_G, float *d_Z, int64_t k, float lr, float momentum, float weight_decay,

@@ -545,10 +545,33 @@ int run_host_step(sgp_handle *h, const StepArgs &a, const float *h_G, float *h_Z
     SGP_CUDA_TRY(h, cudaStreamCreateWithFlags(&h->s_d2h, cudaStreamNonBlocking));
     SGP_CUDA_TRY(h, cudaEventCreateWithFlags(&h->ev_entry, cudaEventDisableTiming));
   }
-  // default chunk: about 64 MB of gradient per chunk, a multiple of 1024 columns
+  // default chunk: about 64 MB of gradient per chunk, a multiple of 1024 columns; the first and last chunks are
+  // smaller (8, 16, 32 MB ...) so that the pipeline fills and drains in a fraction of a chunk time
+  const bool ramp = chunk_cols <= 0;
   if (chunk_cols <= 0) chunk_cols = std::max<int64_t>(1024, (int64_t{64} << 20) / (4 * h->n) / 1024 * 1024);
   chunk_cols = (chunk_cols + 3) / 4 * 4;
-  const int64_t nchunks = (h->d + chunk_cols - 1) / chunk_cols;
+  std::vector<int64_t> bounds{0};
+  if (ramp && h->d >= 4 * chunk_cols) {
+    std::vector<int64_t> head;
+    for (int64_t w = std::max<int64_t>(1024, chunk_cols / 8 / 1024 * 1024); w < chunk_cols; w *= 2) head.push_back(w);
+    int64_t head_cols = 0;
+    for (int64_t w : head) head_cols += w;
+    for (int64_t w : head) bounds.push_back(bounds.back() + w);
+    while (h->d - head_cols - bounds.back() > chunk_cols) bounds.push_back(bounds.back() + chunk_cols);
+    // what is left (at most a chunk plus the tail ramp) goes out in halves down to the smallest head chunk
+    int64_t left = h->d - bounds.back();
+    for (size_t i = head.size(); i-- > 0 && left > head[i];) {
+      const int64_t w = std::max<int64_t>(head[i], (left / 2 + 1023) / 1024 * 1024);
+      if (w >= left) break;
+      bounds.push_back(bounds.back() + w);
+      left -= w;
+    }
+    bounds.push_back(h->d);
+  } else {
+    while (bounds.back() + chunk_cols < h->d) bounds.push_back(bounds.back() + chunk_cols);
+    bounds.push_back(h->d);
+  }
+  const int64_t nchunks = static_cast<int64_t>(bounds.size()) - 1;
   while (static_cast<int64_t>(h->ev_in.size()) < nchunks) {
     cudaEvent_t ev_a = nullptr, ev_b = nullptr;
     SGP_CUDA_TRY(h, cudaEventCreateWithFlags(&ev_a, cudaEventDisableTiming));
@@ -568,7 +591,7 @@ int run_host_step(sgp_handle *h, const StepArgs &a, const float *h_G, float *h_Z
   }
   const size_t pitch = static_cast<size_t>(h->ld) * sizeof(float);
   for (int64_t c = 0; c < nchunks; ++c) {
-    const int64_t c0 = c * chunk_cols, c1 = std::min(h->d, c0 + chunk_cols);
+    const int64_t c0 = bounds[static_cast<size_t>(c)], c1 = bounds[static_cast<size_t>(c) + 1];
     const size_t width = static_cast<size_t>(c1 - c0) * sizeof(float);
     SGP_CUDA_TRY(h, cudaMemcpy2DAsync(d_G + c0, pitch, h_G + c0, pitch, width, static_cast<size_t>(h->n),
                                       cudaMemcpyHostToDevice, h->s_h2d));
