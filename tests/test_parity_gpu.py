@@ -243,6 +243,32 @@ def test_step_host_matches_device_step(binding, inputs):
         assert torch.equal(X, X2) and torch.equal(W, W2) and torch.equal(M, M2)
 
 
+def test_step_host_default_chunking_ramps_and_matches_device_step(binding, inputs):
+    """With the default chunk width the pipeline starts and ends on narrower chunks (n = 256: 8 K, 16 K, 32 K columns,
+    then 64 K): more launches than equal chunks would need, the same bits as the device entry point."""
+    import dataclasses
+    for tau in (0, 1):
+        w = dataclasses.replace(inputs.sweep_workload(256, 300_004), tau=tau, K=2)
+        n, d = w.n, w.d
+        X = inputs.initial_x(w, device=DEV).contiguous(); W = torch.ones(n, device=DEV)
+        M = torch.zeros((n, d), device=DEV); Z = torch.empty((n, d), device=DEV); G = torch.empty((n, d), device=DEV)
+        X2, W2, M2 = X.clone(), W.clone(), M.clone()
+        dG = torch.empty((n, d), device=DEV); dZ = torch.empty((n, d), device=DEV)
+        hG = torch.empty((n, d), pin_memory=True); hZ = torch.empty((n, d), pin_memory=True)
+        with binding.Sgp(n, d, graph_desc(w, binding), tau=tau) as h1, binding.Sgp(n, d, graph_desc(w, binding), tau=tau) as h2:
+            for k in range(w.K):
+                inputs.gradient(w, k, G)
+                hG.copy_(G)
+                h1.step(X, W, M, G, Z, k, w.lr, w.momentum, 0.0, True)
+                torch.cuda.synchronize()
+                before = h2.get_option("launches")
+                h2.step_host(X2, W2, M2, hG, hZ, dG, dZ, k, w.lr, w.momentum, 0.0, True)
+                assert h2.get_option("launches") - before >= 8          # equal 64 K chunks would be 5
+                assert torch.equal(hZ, Z.cpu())
+            assert h2.device_status() == 0
+        assert torch.equal(X, X2) and torch.equal(W, W2) and torch.equal(M, M2)
+
+
 def test_invalid_step_arguments(binding, inputs):
     n, d = 4, 64
     X = torch.zeros((n, d), device=DEV); W = torch.ones(n, device=DEV); G = torch.zeros((n, d), device=DEV)
