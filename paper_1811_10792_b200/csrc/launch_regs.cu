@@ -24,14 +24,15 @@ inline int floor_log2(int64_t v) {
 
 }  // namespace
 
-template <> RegsKernel regs_kernel_of<4, false>(int, bool, bool);
-template <> RegsKernel regs_kernel_of<4, true>(int, bool, bool);
-template <> RegsKernel regs_kernel_of<1, false>(int, bool, bool);
-template <> RegsKernel regs_kernel_of<1, true>(int, bool, bool);
+template <> RegsKernel regs_kernel_of<4, false>(int, bool, bool, bool);
+template <> RegsKernel regs_kernel_of<4, true>(int, bool, bool, bool);
+template <> RegsKernel regs_kernel_of<1, false>(int, bool, bool, bool);
+template <> RegsKernel regs_kernel_of<1, true>(int, bool, bool, bool);
 
-RegsKernel regs_kernel(int vec, int upd, bool has_z, bool has_ring, bool diag) {
-  if (vec == 4) return diag ? regs_kernel_of<4, true>(upd, has_z, has_ring) : regs_kernel_of<4, false>(upd, has_z, has_ring);
-  return diag ? regs_kernel_of<1, true>(upd, has_z, has_ring) : regs_kernel_of<1, false>(upd, has_z, has_ring);
+RegsKernel regs_kernel(int vec, int upd, bool has_z, bool has_ring, bool diag, bool gather_first) {
+  if (vec == 4)
+    return diag ? regs_kernel_of<4, true>(upd, has_z, has_ring, gather_first) : regs_kernel_of<4, false>(upd, has_z, has_ring, gather_first);
+  return diag ? regs_kernel_of<1, true>(upd, has_z, has_ring, gather_first) : regs_kernel_of<1, false>(upd, has_z, has_ring, gather_first);
 }
 
 int kernel_info(int device, const void *kern, size_t smem, KernelInfo *out, int *cuda_error) {
@@ -145,7 +146,12 @@ int launch_regs(const DeviceInfo &dev, StepParams p, const ConstTable *ct, int u
   p.log2_tile_vecs = floor_log2(tv);
   const int64_t tile_cols = tv * vec;
   const int64_t ntiles = (ncols + tile_cols - 1) / tile_cols;
-  RegsKernel kern = regs_kernel(vec, upd, p.Z != nullptr, has_ring, p.diag != nullptr);
+  // Order of instructions inside a phase (momentum updates without a ring): every gather of a batch before its
+  // stores wins where the tile is made of full four-item batches and row segments are at least 512 bytes (n = 4..96:
+  // +1 to +1.7 % of the copy bandwidth) and loses elsewhere (n = 24, three-item batches: 0.935 against 0.974; ragged
+  // last batch, n = 104, 112: 0.89 against 0.92-0.93; 256-byte segments, n = 128, 256: 0.91 against 0.93).
+  const bool gather_first = (static_cast<int64_t>(n) * tv) % (4 * kThreads) == 0 && tile_cols * 4 >= 512;
+  RegsKernel kern = regs_kernel(vec, upd, p.Z != nullptr, has_ring, p.diag != nullptr, gather_first);
   KernelInfo ki;
   {
     const int rc = kernel_info(dev.device, reinterpret_cast<const void *>(kern), smem, &ki, &rec->cuda_error);

@@ -7,7 +7,7 @@
 
 namespace sgp {
 
-template <int VEC, int UPD, bool HAS_Z, bool HAS_RING, bool DIAG>
+template <int VEC, int UPD, bool HAS_Z, bool HAS_RING, bool DIAG, bool GATHER_FIRST>
 __global__ void __launch_bounds__(kThreads, 2)
 sgp_step_regs_kernel(const __grid_constant__ StepParams p, const __grid_constant__ ConstTable ct) {
   using V = typename VecT<VEC>::type;
@@ -17,8 +17,11 @@ sgp_step_regs_kernel(const __grid_constant__ StepParams p, const __grid_constant
   // of the copy bandwidth, and with diagnostics on top it spills
   constexpr int kItemsPerThread = (UPD == kUpdAdam && HAS_RING) ? 3 : UpdTraits<UPD>::kItems;
   constexpr int kDiagArrays = HAS_RING ? 2 : 1;
-  // plain SGD (8 items per thread) loses with this ordering: 0.85 against 0.95
-  constexpr bool kGatherFirst = !HAS_RING && (UPD == kUpdHeavyBall || UPD == kUpdNesterov);
+  // GATHER_FIRST (momentum updates without a ring only; the launcher picks it for tiles made of full four-item batches
+  // with row segments of 512 bytes or more): every gather of a batch before its stores, every update before its
+  // momentum stores.  Plain SGD (8 items per thread) loses with this ordering: 0.85 against 0.95.
+  constexpr bool kGatherFirst = GATHER_FIRST;
+  static_assert(!GATHER_FIRST || (!HAS_RING && (UPD == kUpdHeavyBall || UPD == kUpdNesterov)), "not instantiated");
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int n = p.n;
   const int tv = 1 << p.log2_tile_vecs;
@@ -260,7 +263,8 @@ sgp_step_regs_kernel(const __grid_constant__ StepParams p, const __grid_constant
 using RegsKernel = void (*)(const StepParams, const ConstTable);
 // The instantiation for (vector width 4 or 1, optimiser, Z written, delay ring, fused diagnostics); the kernels are
 // spread over several translation units so that they compile in parallel.
-RegsKernel regs_kernel(int vec, int upd, bool has_z, bool has_ring, bool diag);
-template <int VEC, bool DIAG> RegsKernel regs_kernel_of(int upd, bool has_z, bool has_ring);
+// gather_first is honoured for momentum updates without a ring and ignored elsewhere.
+RegsKernel regs_kernel(int vec, int upd, bool has_z, bool has_ring, bool diag, bool gather_first);
+template <int VEC, bool DIAG> RegsKernel regs_kernel_of(int upd, bool has_z, bool has_ring, bool gather_first);
 
 }  // namespace sgp
