@@ -35,7 +35,7 @@ struct LaunchRecord {
 struct KernelInfo {
   int num_regs = 0;
   size_t static_smem = 0;
-  size_t enabled_smem = 48 * 1024;
+  size_t enabled_smem = 48 * 1024;   // largest DYNAMIC size a launch may ask for (48 KB less the static part at first)
 };
 int kernel_info(int device, const void *kern, size_t smem, KernelInfo *out, int *cuda_error);
 // Clusters of `cluster` CTAs (kThreads threads, `smem` dynamic bytes each) of `kern` that `device` holds at once;

@@ -47,6 +47,8 @@ int kernel_info(int device, const void *kern, size_t smem, KernelInfo *out, int 
       KernelInfo ki;
       ki.num_regs = fa.numRegs;
       ki.static_smem = fa.sharedSizeBytes;
+      // without the attribute a launch may use 48 KB of shared memory, static part included
+      ki.enabled_smem = 48 * 1024 - std::min<size_t>(48 * 1024, fa.sharedSizeBytes);
       it = g_kernel_info.emplace(key, ki).first;
     }
   }

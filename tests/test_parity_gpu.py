@@ -500,6 +500,36 @@ def test_cluster_kernel_matches_oracle_and_register_kernel(binding, inputs, n, d
         assert np.array_equal(a[name], b[name]), name
 
 
+def test_dynamic_shared_memory_just_under_48_kb(binding, inputs):
+    """n = 88 with the sweep's tenth graph needs 49,148 bytes of dynamic shared memory: with the kernel's few static
+    bytes that is over the 48 KB a launch gets without the opt-in attribute (the launch used to fail with
+    cudaErrorInvalidValue on exactly that step)."""
+    w = dataclasses.replace(inputs.sweep_workload(88, 3_000), K=12)
+    out = _run_gpu(binding, inputs, w, options={"variant": 1})
+    _compare(w, out)
+
+
+@pytest.mark.parametrize("tau,diag", [(0, 0), (1, 0), (0, 1), (2, 1)])
+def test_every_node_count_launches(binding, inputs, tau, diag):
+    """Every n from 1 to 256 on the sweep's ten random digraphs (table sizes, tile widths and shared-memory sizes all
+    differ), with and without a delay ring and the fused diagnostics: no launch fails, no status bit, the weights
+    (ring included) still sum to n."""
+    d = 1_030
+    for n in range(1, 257):
+        w = inputs.sweep_workload(n, d)
+        X = torch.zeros((n, d), device=DEV); M = torch.zeros((n, d), device=DEV); Z = torch.empty((n, d), device=DEV)
+        G = torch.ones((n, d), device=DEV); W = torch.ones(n, device=DEV)
+        with binding.Sgp(n, d, graph_desc(w, binding), tau=tau) as h:
+            h.set_option("diagnostics", diag)
+            for k in range(10):
+                h.step(X, W, M, G, Z, k, w.lr, w.momentum, 0.0, True)
+            torch.cuda.synchronize()
+            assert h.device_status() == 0, n
+            stats = h.check(X, W)
+            assert stats["code"] == binding.SGP_OK and abs(stats["sum_w"] - n) < 1e-4 * n, (n, stats)
+        assert torch.isfinite(X).all() and torch.isfinite(Z).all(), n
+
+
 # ------------------------------------------------------------------ lockstep clusters of the register-staged kernel
 @pytest.mark.parametrize("n,d,tau,size,diag", [(32, 1_029, 0, 2, 0), (32, 70_001, 1, 2, 0), (64, 9_003, 0, 4, 0), (5, 2_000, 2, 4, 0),
                                                (130, 2_052, 0, 4, 0), (2, 260, 0, 2, 0), (48, 40_000, 1, 2, 1), (8, 300_001, 0, 4, 1)])
