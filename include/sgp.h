@@ -350,7 +350,9 @@ int sgp_step_static(int n, int64_t d, int64_t ld, const int32_t *h_rowptr, const
  *              the receiver applies p_ij, so all out-neighbours of a node read the same slot
  *     tau >= 1 : the messages consumed at step k were published at step k - tau, so update + pull + mix are ONE
  *              kernel per step (sgp_rank_step_overlap) and the exchange never waits.
- * Results are bit-identical to sgp_step on the stacked n x d arrays (same CSR order, same FMA chain).
+ * Results are bit-identical to sgp_step on the stacked n x d arrays (same CSR order, same FMA chain); the one
+ * exception is sgp_step's shortcut for steps whose rows of P are all alike with tau == 0 (complete graph), which sums
+ * interleaved partial sums: there the two agree to rounding, not bit for bit.
  *
  * Synchronisation is the caller's (one barrier per step across the ranks, e.g. an all-reduce of one element on the
  * step's stream): tau == 0: update, BARRIER, mix; tau >= 1: step_overlap, BARRIER.  No kernel of this library

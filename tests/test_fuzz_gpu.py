@@ -5,6 +5,7 @@ import numpy as np
 import pytest
 
 from gpu_runner import compare_with_oracle, run_gpu
+from parity_util import assert_close, oracle_P_of_k
 
 
 @pytest.fixture(scope="module")
@@ -68,3 +69,67 @@ def test_draws_cover_the_space():
     assert {c["opts"]["lockstep"] for c in draws} == {0, 1, 2, 4}
     assert any(c["pad"] % 4 for c in draws) and any(c["offset"] % 4 for c in draws)
     assert min(c["n"] for c in draws) <= 2 and max(c["n"] for c in draws) >= 128
+
+
+def _draw_adam(case: int):
+    rng = np.random.RandomState(9_1811 + case)
+    n = int(np.clip(np.round(2.0 ** rng.uniform(0.0, 8.0)), 1, 256))
+    graph = rng.choice(["exp", "exp2", "random", "complete"], p=[0.35, 0.2, 0.35, 0.1])
+    d = int(rng.choice([rng.randint(1, 40), rng.randint(40, 700), rng.randint(700, 5000)]))
+    opts = {"variant": int(rng.choice([0, 0, 1, 3])), "lockstep": int(rng.choice([0, 1, 2]))}
+    return dict(n=n, d=d, tau=int(rng.choice([0, 0, 1, 2])), graph=graph, K=int(rng.randint(3, 7)),
+                pad=int(rng.choice([0, 0, 2, 4])), offset=int(rng.choice([0, 0, 1, 4])), write_z=bool(rng.rand() < 0.8),
+                wd=float(rng.choice([0.0, 1e-2])), opts=opts, seed=int(rng.randint(1, 1 << 30)))
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("case", range(64))
+def test_random_adam_configuration_matches_oracle(binding, inputs, case):
+    """The same for the Adam-preconditioned step (Sec. 6.2 / App. C.1)."""
+    from test_adam_gpu import _compare as adam_compare, _run as adam_run
+    c = _draw_adam(case)
+    kind, peers = ("exp", 2) if c["graph"] == "exp2" else (c["graph"], 1)
+    w = inputs.Workload(f"fuzz_adam{case}", n=c["n"], d=c["d"], K=c["K"], graph=kind, peers=peers, max_outdeg=4,
+                        num_steps=5, tau=c["tau"], seed=c["seed"], optimizer="adam")
+    out = adam_run(binding, inputs, w, options=c["opts"], ld=c["d"] + c["pad"], offset=c["offset"], wd=c["wd"],
+                   write_z=c["write_z"])
+    adam_compare(w, out, wd=c["wd"], write_z=c["write_z"])
+
+
+def _draw_rank(case: int):
+    rng = np.random.RandomState(7_1811 + case)
+    n = int(np.clip(np.round(2.0 ** rng.uniform(0.0, 5.3)), 1, 40))
+    graph = rng.choice(["exp", "exp2", "random", "complete", "bipartite"], p=[0.3, 0.2, 0.3, 0.1, 0.1])
+    if graph == "bipartite" and n % 2:
+        n += 1
+    if graph == "complete":
+        n = min(n, 32)                       # a mix takes at most 32 sources in this mode
+    return dict(n=n, d=int(rng.choice([rng.randint(1, 40), rng.randint(40, 3000)])), tau=int(rng.choice([0, 0, 1, 2, 3])),
+                graph=graph, momentum=float(rng.choice([0.0, 0.9])), nesterov=bool(rng.rand() < 0.6),
+                offset=int(rng.choice([0, 0, 0, 1, 2])), write_z=bool(rng.rand() < 0.8), K=int(rng.randint(3, 7)),
+                seed=int(rng.randint(1, 1 << 30)))
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("case", range(64))
+def test_random_one_node_per_gpu_configuration_equals_stacked_step(binding, inputs, case):
+    """The split kernels (update / pull + mix, fused overlap step) in loopback give the stacked step's bits
+    (App. C setting, Alg. 1 lines 4-8, Alg. 2), whatever the shape, delay, graph and alignment."""
+    import torch
+    from test_rowshard_gpu import _run_both
+    c = _draw_rank(case)
+    kind, peers = ("exp", 2) if c["graph"] == "exp2" else (c["graph"], 1)
+    w = inputs.Workload(f"fuzz_rank{case}", n=c["n"], d=c["d"], K=c["K"], graph=kind, peers=peers, max_outdeg=4,
+                        num_steps=5, lr=0.05, momentum=c["momentum"], nesterov=c["nesterov"], weight_decay=1e-3,
+                        tau=c["tau"], seed=c["seed"])
+    _x0, _grads, got, stacked = _run_both(binding, inputs, w, c["K"], offset=c["offset"], write_z=c["write_z"])
+    names = ("X", "W") + (("Z",) if c["write_z"] else ()) + (("M",) if c["momentum"] else ())
+    # where every row of a step's matrix is the same (complete graph, or n = 3 with two peers) and tau = 0, the stacked
+    # step sums interleaved partial sums: equal to rounding, not bit for bit
+    P_of_k = oracle_P_of_k(w)
+    shortcut = c["tau"] == 0 and any(bool(np.all(P_of_k(k) == P_of_k(k)[0])) for k in range(c["K"])) and c["n"] > 1
+    for name in names:
+        if shortcut:
+            assert_close(name, got[name].cpu().numpy(), stacked[name].cpu().numpy().astype(np.float64))
+        else:
+            assert torch.equal(got[name], stacked[name]), f"{name}: one-node-per-GPU and stacked results differ"
