@@ -107,6 +107,11 @@ int64_t regs_tile_cols(int n, size_t fixed) {
   const size_t copies = auto_single_buffer(n) ? 1 : 2;
   const size_t cap = (copies == 1 ? 88 : 80) * 1024;     // n = 80 at 85 KB: 0.97; n = 96 at 102 KB: 0.79
   while (cols > 32 && copies * static_cast<size_t>(n) * cols * 4 + fixed > cap) cols >>= 1;
+  // Between four and six items per thread the tile falls into a batch of three and a batch of one to three (n = 5,
+  // 10, 20: 0.92-0.93 of the copy bandwidth where the neighbours reach 0.98): twice the width in ONE exchange tile
+  // (the same shared memory) gives three fuller batches instead (0.99).
+  const int64_t items = static_cast<int64_t>(n) * cols / 4;
+  if (copies == 2 && items > 4 * kThreads && items < 6 * kThreads) cols *= 2;
   return cols;
 }
 
@@ -129,7 +134,8 @@ int launch_regs(const DeviceInfo &dev, StepParams p, const ConstTable *ct, int u
   else p.table_mode = table_bytes <= 40 * 1024 ? 1 : 2;
   const bool uniform = !has_ring && uniform_rows;
   // large n: one exchange tile (two barriers per tile) so that the row segments can stay twice as long
-  p.single_buffer = opt.single_buffer == 1 ? 1 : (opt.single_buffer == 2 ? 0 : (auto_single_buffer(n) ? 1 : 0));
+  // (also for the doubled tiles of regs_tile_cols: more than eight items per thread at n <= 32)
+  p.single_buffer = opt.single_buffer == 1 ? 1 : (opt.single_buffer == 2 ? 0 : ((auto_single_buffer(n) || (n <= 32 && n * tv > 8 * kThreads)) ? 1 : 0));
   // diagnostics add up to 32 KB of scratch: one exchange tile then keeps the CTA's footprint (and with it the
   // share of the SM left to the L1) where it was (tau = 1, n = 32: 96 KB per CTA ran at 0.67, 64 KB does not)
   if (p.diag != nullptr && opt.single_buffer == 0) p.single_buffer = 1;
