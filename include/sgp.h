@@ -379,6 +379,11 @@ typedef struct sgp_rank_plan_t {
   float   weight[SGP_RANK_MAX_SOURCES];
 } sgp_rank_plan_t;
 int sgp_rank_plan(const sgp_schedule *s, int rank, int64_t k, int tau, sgp_rank_plan_t *out);
+/* The same with a send period s >= 1 (Alg. 2 line 5; the stacked path's "send_period" option): nodes transmit only on
+ * steps k with k mod s == 0, and the c-th transmission (k = c s) uses P^(c).  On every other step the matrix is the
+ * identity: self_weight = 1 and, for tau == 0, the list holds the node itself alone; for tau >= 1 the list is empty
+ * unless step k - tau was a transmission, whose off-diagonal row then arrives.  send_period == 1 is sgp_rank_plan. */
+int sgp_rank_plan_period(const sgp_schedule *s, int rank, int64_t k, int tau, int64_t send_period, sgp_rank_plan_t *out);
 
 /* Creates rank `rank` of `world` on the current device: compiles the schedule for n = world nodes and allocates
  * and zeroes (tau + 2) message slots of d (+ padding) floats.  Synchronises. */
@@ -391,6 +396,9 @@ int sgp_rank_message_block(sgp_rank *r, void **d_block, size_t *bytes);
 /* d_peer_blocks[j] (HOST array of `world` device pointers valid in this process; entry [rank] is ignored, entries
  * of ranks this node never receives from may be NULL): where rank j's message block is mapped. */
 int sgp_rank_set_peers(sgp_rank *r, void *const *d_peer_blocks);
+/* Send period of this rank's steps (default 1, at most 2^20); every rank of a run must set the same value before
+ * the first step. */
+int sgp_rank_set_send_period(sgp_rank *r, int64_t send_period);
 /* tau == 0, first half: publishes (h, w) of step k; m updated in place; x untouched.  Asynchronous. */
 int sgp_rank_update(sgp_rank *r, const float *d_x, float *d_w, float *d_m, const float *d_g, int64_t k, float lr,
                     float momentum, float weight_decay, int nesterov, void *stream);

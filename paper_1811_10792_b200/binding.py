@@ -35,7 +35,7 @@ EXPORTS = [
     "sgp_rank_plan", "sgp_rank_create", "sgp_rank_destroy", "sgp_rank_get_schedule", "sgp_rank_message_block",
     "sgp_rank_set_peers", "sgp_rank_update", "sgp_rank_mix", "sgp_rank_step_overlap", "sgp_rank_device_status",
     "sgp_ipc_export", "sgp_ipc_open", "sgp_ipc_close", "sgp_step_adam_host", "sgp_rank_update_adam",
-    "sgp_rank_step_overlap_adam",
+    "sgp_rank_step_overlap_adam", "sgp_rank_plan_period", "sgp_rank_set_send_period",
 ]
 SGP_RANK_MAX_SOURCES = 32
 SGP_IPC_HANDLE_BYTES = 64
@@ -97,6 +97,8 @@ def _load() -> C.CDLL:
         "sgp_last_cuda_error": [vp],
         "sgp_version": [],
         "sgp_rank_plan": [vp, i32, i64, i32, C.POINTER(sgp_rank_plan_t)],
+        "sgp_rank_plan_period": [vp, i32, i64, i32, i64, C.POINTER(sgp_rank_plan_t)],
+        "sgp_rank_set_send_period": [vp, i64],
         "sgp_rank_create": [C.POINTER(vp), i32, i32, i64, C.POINTER(sgp_graph_desc), i32, C.c_uint],
         "sgp_rank_destroy": [vp],
         "sgp_rank_get_schedule": [vp, C.POINTER(vp)],
@@ -208,10 +210,14 @@ class _ScheduleView:
         return rowptr, col[:nnz], val[:nnz]
 
 
-def rank_plan(schedule: "_ScheduleView", rank: int, k: int, tau: int) -> dict:
-    """sgp_rank_plan (host only): what `rank` publishes and pulls at step k in the one-node-per-GPU mode."""
+def rank_plan(schedule: "_ScheduleView", rank: int, k: int, tau: int, send_period: int = 1) -> dict:
+    """sgp_rank_plan / sgp_rank_plan_period (host only): what `rank` publishes and pulls at step k in the
+    one-node-per-GPU mode."""
     out = sgp_rank_plan_t()
-    _check(_lib.sgp_rank_plan(schedule._ptr, rank, k, tau, C.byref(out)), "sgp_rank_plan")
+    if send_period == 1:
+        _check(_lib.sgp_rank_plan(schedule._ptr, rank, k, tau, C.byref(out)), "sgp_rank_plan")
+    else:
+        _check(_lib.sgp_rank_plan_period(schedule._ptr, rank, k, tau, send_period, C.byref(out)), "sgp_rank_plan_period")
     return dict(write_slot=out.write_slot, read_slot=out.read_slot, self_weight=np.float32(out.self_weight),
                 self_pos=out.self_pos, senders=[out.sender[e] for e in range(out.count)],
                 weights=np.array([out.weight[e] for e in range(out.count)], dtype=np.float32))
@@ -422,6 +428,10 @@ class SgpRank:
         ptr, size = C.c_void_p(), C.c_size_t()
         _check(_lib.sgp_rank_message_block(self._h, C.byref(ptr), C.byref(size)), "sgp_rank_message_block")
         return ptr.value, size.value
+
+    def set_send_period(self, send_period: int) -> None:
+        """Nodes transmit only on steps k with k mod send_period == 0 (Alg. 2 line 5); every rank must set the same."""
+        _check(_lib.sgp_rank_set_send_period(self._h, send_period), "sgp_rank_set_send_period")
 
     def set_peers(self, pointers) -> None:
         """pointers[j]: device address (int or None) of rank j's message block in this process."""

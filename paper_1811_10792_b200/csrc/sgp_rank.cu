@@ -22,6 +22,7 @@ struct sgp_rank {
   std::vector<const float *> peer_block;  // where every rank's block is mapped in this process
   unsigned *d_words = nullptr;            // [0] ticket, [1] status
   int last_cuda_error = 0;
+  int64_t send_period = 1;                // nodes transmit on steps k with k mod send_period == 0 (Alg. 2 line 5)
 };
 
 namespace {
@@ -94,35 +95,49 @@ void fill_params(const sgp_rank *r, sgp::RankParams *p) {
 
 extern "C" {
 
-int sgp_rank_plan(const sgp_schedule *s, int rank, int64_t k, int tau, sgp_rank_plan_t *out) {
-  if (s == nullptr || out == nullptr || rank < 0 || rank >= s->n || k < 0 || tau < 0 || tau > 64) return SGP_ERR_ARG;
+int sgp_rank_plan_period(const sgp_schedule *s, int rank, int64_t k, int tau, int64_t send_period, sgp_rank_plan_t *out) {
+  if (s == nullptr || out == nullptr || rank < 0 || rank >= s->n || k < 0 || tau < 0 || tau > 64 || send_period < 1)
+    return SGP_ERR_ARG;
   sgp_rank_plan_t plan;
   std::memset(&plan, 0, sizeof(plan));
   const int slots = tau + 2;
   plan.write_slot = static_cast<int32_t>(k % slots);
   plan.self_pos = -1;
-  {
+  // Matrix of step kk: the c-th transmission (kk = c * send_period) uses P^(c); a step on which nobody transmits
+  // mixes with the identity (Alg. 2 lines 5-12).
+  const bool sends_now = k % send_period == 0;
+  const int64_t k_arrive = k - tau;                       // the step whose messages arrive now
+  const bool arrives = tau == 0 ? sends_now : (k_arrive >= 0 && k_arrive % send_period == 0);
+  plan.self_weight = 1.0f;
+  if (sends_now) {
     // the self weight is this step's p_ii
-    const SgpStepCsr &now = s->slot(k);
+    const SgpStepCsr &now = s->slot(k / send_period);
     for (int32_t e = now.rowptr[static_cast<size_t>(rank)]; e < now.rowptr[static_cast<size_t>(rank) + 1]; ++e)
       if (now.col[static_cast<size_t>(e)] == rank) plan.self_weight = now.val[static_cast<size_t>(e)];
   }
   if (tau == 0) {
     plan.read_slot = plan.write_slot;
-    const SgpStepCsr &c = s->slot(k);
-    const int32_t b = c.rowptr[static_cast<size_t>(rank)], e1 = c.rowptr[static_cast<size_t>(rank) + 1];
-    if (e1 - b > SGP_RANK_MAX_SOURCES) return SGP_ERR_ARG;
-    for (int32_t e = b; e < e1; ++e) {
-      if (c.col[static_cast<size_t>(e)] == rank) plan.self_pos = plan.count;
-      plan.sender[plan.count] = c.col[static_cast<size_t>(e)];
-      plan.weight[plan.count] = c.val[static_cast<size_t>(e)];
-      ++plan.count;
+    if (arrives) {
+      const SgpStepCsr &c = s->slot(k / send_period);
+      const int32_t b = c.rowptr[static_cast<size_t>(rank)], e1 = c.rowptr[static_cast<size_t>(rank) + 1];
+      if (e1 - b > SGP_RANK_MAX_SOURCES) return SGP_ERR_ARG;
+      for (int32_t e = b; e < e1; ++e) {
+        if (c.col[static_cast<size_t>(e)] == rank) plan.self_pos = plan.count;
+        plan.sender[plan.count] = c.col[static_cast<size_t>(e)];
+        plan.weight[plan.count] = c.val[static_cast<size_t>(e)];
+        ++plan.count;
+      }
+    } else {
+      plan.self_pos = 0;                                   // identity: the node keeps its whole half step
+      plan.sender[0] = rank;
+      plan.weight[0] = 1.0f;
+      plan.count = 1;
     }
   } else {
     plan.read_slot = static_cast<int32_t>(((k - tau) % slots + slots) % slots);
-    if (k >= tau) {
+    if (arrives) {
       // the messages that arrive now were sent, and weighted, with the matrix of step k - tau
-      const SgpStepCsr &c = s->slot(k - tau);
+      const SgpStepCsr &c = s->slot(k_arrive / send_period);
       const int32_t b = c.rowptr[static_cast<size_t>(rank)], e1 = c.rowptr[static_cast<size_t>(rank) + 1];
       if (e1 - b - 1 > SGP_RANK_MAX_SOURCES) return SGP_ERR_ARG;
       for (int32_t e = b; e < e1; ++e) {
@@ -134,6 +149,16 @@ int sgp_rank_plan(const sgp_schedule *s, int rank, int64_t k, int tau, sgp_rank_
     }
   }
   *out = plan;
+  return SGP_OK;
+}
+
+int sgp_rank_plan(const sgp_schedule *s, int rank, int64_t k, int tau, sgp_rank_plan_t *out) {
+  return sgp_rank_plan_period(s, rank, k, tau, 1, out);
+}
+
+int sgp_rank_set_send_period(sgp_rank *r, int64_t send_period) {
+  if (r == nullptr || send_period < 1 || send_period > (1 << 20)) return SGP_ERR_ARG;
+  r->send_period = send_period;
   return SGP_OK;
 }
 
@@ -265,7 +290,7 @@ int rank_overlap(sgp_rank *r, float *d_x, float *d_w, float *d_m, float *d_v, co
   int rc = check_device(r);
   if (rc != SGP_OK) return rc;
   sgp_rank_plan_t plan;
-  rc = sgp_rank_plan(r->sched, r->rank, k, r->tau, &plan);
+  rc = sgp_rank_plan_period(r->sched, r->rank, k, r->tau, r->send_period, &plan);
   if (rc != SGP_OK) return rc;
   sgp::RankSources s;
   rc = make_sources(r, plan, &s);
@@ -327,7 +352,7 @@ int sgp_rank_mix(sgp_rank *r, float *d_x, float *d_w, float *d_z, int64_t k, voi
   int rc = check_device(r);
   if (rc != SGP_OK) return rc;
   sgp_rank_plan_t plan;
-  rc = sgp_rank_plan(r->sched, r->rank, k, 0, &plan);
+  rc = sgp_rank_plan_period(r->sched, r->rank, k, 0, r->send_period, &plan);
   if (rc != SGP_OK) return rc;
   sgp::RankSources s;
   rc = make_sources(r, plan, &s);

@@ -30,9 +30,12 @@ def step_protocol(tau: int):
 class LoopbackGroup:
     """``world`` virtual ranks on the current device of this process."""
 
-    def __init__(self, world: int, d: int, graph: binding.GraphDesc, tau: int = 0, flags: int = 0):
+    def __init__(self, world: int, d: int, graph: binding.GraphDesc, tau: int = 0, flags: int = 0, send_period: int = 1):
         self.world, self.d, self.tau = world, d, tau
         self.ranks = [binding.SgpRank(r, world, d, graph, tau=tau, flags=flags) for r in range(world)]
+        if send_period != 1:
+            for rk in self.ranks:
+                rk.set_send_period(send_period)
         blocks = [rk.message_block()[0] for rk in self.ranks]
         for rk in self.ranks:
             rk.set_peers(blocks)
@@ -98,7 +101,8 @@ def exchange_handles(rank: int, world: int, my_handle: bytes, group=None):
 class DistributedRank:
     """This process's node under torch.distributed (one process per GPU, all GPUs in one NVLink domain)."""
 
-    def __init__(self, d: int, graph: binding.GraphDesc, tau: int = 0, flags: int = 0, group=None, device=None):
+    def __init__(self, d: int, graph: binding.GraphDesc, tau: int = 0, flags: int = 0, group=None, device=None,
+                 send_period: int = 1):
         import torch
         import torch.distributed as dist
         self.group = group
@@ -106,6 +110,8 @@ class DistributedRank:
         self.tau = tau
         self.device = torch.device("cuda", torch.cuda.current_device()) if device is None else device
         self.node = binding.SgpRank(self.rank, self.world, d, graph, tau=tau, flags=flags)
+        if send_period != 1:
+            self.node.set_send_period(send_period)
         ptr, _ = self.node.message_block()
         handles = exchange_handles(self.rank, self.world, binding.ipc_export(ptr), group=group)
         self._mapped = []

@@ -28,7 +28,7 @@ def inputs():
     return i
 
 
-def _run_both(binding, inputs, w, K, offset=0, write_z=True, flags=0):
+def _run_both(binding, inputs, w, K, offset=0, write_z=True, flags=0, send_period=1):
     """K steps in loopback one-node-per-GPU mode and K steps of the stacked step on the same inputs."""
     from paper_1811_10792_b200 import rowshard
     n, d = w.n, w.d
@@ -49,7 +49,8 @@ def _run_both(binding, inputs, w, K, offset=0, write_z=True, flags=0):
         ms[r][1].zero_()
     grads = []
     with binding.Sgp(n, d, graph_desc(w, binding), tau=w.tau, flags=flags) as h, \
-            rowshard.LoopbackGroup(n, d, graph_desc(w, binding), tau=w.tau, flags=flags) as grp:
+            rowshard.LoopbackGroup(n, d, graph_desc(w, binding), tau=w.tau, flags=flags, send_period=send_period) as grp:
+        h.set_option("send_period", send_period)
         for k in range(K):
             inputs.gradient(w, k, G)
             grads.append(G.cpu().numpy().astype(np.float64))
@@ -104,6 +105,22 @@ def test_loopback_ranks_match_oracle_and_stacked_step(binding, inputs, case):
         assert torch.equal(got[name], stacked[name]), f"{name}: one-node-per-GPU and stacked results differ"
     if case["graph"] == "random":
         assert np.ptp(got["W"].cpu().numpy()) > 1e-3                    # the weight path is exercised
+
+
+@pytest.mark.parametrize("n,graph,tau,period", [(8, "exp", 0, 2), (8, "exp", 1, 2), (8, "exp", 2, 2), (12, "random", 1, 3),
+                                                (12, "random", 0, 3), (16, "exp", 3, 4)])
+def test_loopback_with_a_send_period(binding, inputs, n, graph, tau, period):
+    """Alg. 2 line 5 in the one-node-per-GPU mode: transmissions only every `period` steps, identity mixing in between;
+    the oracle's recursion with the same send period, and the stacked step's bits."""
+    from oracle import sgp as osgp
+    w = dataclasses.replace(inputs.sweep_workload(n, 1_503), graph=graph, peers=1, tau=tau, weight_decay=1e-3)
+    K = 9
+    x0, grads, got, stacked = _run_both(binding, inputs, w, K, send_period=period)
+    st = osgp.sgp_run(x0, K, oracle_P_of_k(w), lambda k, z: grads[k], w.lr, momentum=w.momentum, nesterov=w.nesterov,
+                      weight_decay=w.weight_decay, tau=w.tau, send_period=period)
+    for name, want in (("X", st.x), ("Z", st.z), ("W", st.w), ("M", st.u)):
+        assert_close(name, got[name].cpu().numpy(), want)
+        assert torch.equal(got[name], stacked[name]), f"{name}: one-node-per-GPU and stacked results differ"
 
 
 def test_loopback_without_z_and_biased(binding, inputs):

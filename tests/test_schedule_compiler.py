@@ -226,6 +226,56 @@ def test_rank_plan_host_only(binding):
         assert e.value.code == binding.SGP_ERR_ARG
 
 
+@pytest.mark.parametrize("n,kind,tau,period", [(8, "exp1", 0, 2), (8, "exp1", 1, 2), (8, "exp2", 2, 2), (6, "random", 1, 3),
+                                               (6, "random", 0, 3), (16, "exp1", 3, 4), (5, "random", 2, 1)])
+def test_rank_plans_with_a_send_period_reproduce_the_oracle_recursion(binding, n, kind, tau, period):
+    """sgp_rank_plan_period (host only): all ranks emulated in one process -- each publishes its half step into slot
+    write_slot, then mixes what its plan says -- end on the oracle's state for the same send period (Alg. 2 line 5:
+    transmissions only on steps k with k mod s = 0; identity mixing in between; messages arrive tau steps later)."""
+    from oracle import schedule as osched
+    from oracle import sgp as osgp
+    graph = {"exp1": binding.GraphDesc.exp_peers(1), "exp2": binding.GraphDesc.exp_peers(2),
+             "random": binding.GraphDesc.random_outdeg(11, 4, 3)}[kind]
+    okind = dict(exp1=("exp", dict(peers=1)), exp2=("exp", dict(peers=2)),
+                 random=("random", dict(seed=11, max_outdeg=3, num_steps=4)))[kind]
+    P_of_k = lambda k: osched.mixing_matrix(okind[0], n, k, **okind[1])
+    K, d, lr = 11, 5, 0.1
+    rng = np.random.default_rng(5)
+    x = rng.standard_normal((n, d))
+    grads = rng.standard_normal((K, n, d))
+    w = np.ones(n)
+    slots = tau + 2
+    slot_x = np.zeros((n, slots, d))
+    slot_w = np.zeros((n, slots))
+    sched = binding.Schedule(n, graph)
+    for k in range(K):
+        plans = [binding.rank_plan(sched, r, k, tau, send_period=period) for r in range(n)]
+        h = x - lr * grads[k]
+        for r in range(n):                                   # every rank publishes (the barrier comes after this loop)
+            slot_x[r, plans[r]["write_slot"]] = h[r]
+            slot_w[r, plans[r]["write_slot"]] = w[r]
+        new_x, new_w = np.zeros_like(x), np.zeros_like(w)
+        for r, plan in enumerate(plans):
+            if tau > 0:
+                new_x[r] = float(plan["self_weight"]) * h[r]
+                new_w[r] = float(plan["self_weight"]) * w[r]
+                assert plan["self_pos"] == -1
+                if k % period:
+                    assert plan["self_weight"] == np.float32(1.0)
+            for e, j in enumerate(plan["senders"]):
+                new_x[r] += float(plan["weights"][e]) * slot_x[j, plan["read_slot"]]
+                new_w[r] += float(plan["weights"][e]) * slot_w[j, plan["read_slot"]]
+            if tau == 0 and k % period:
+                assert plan["senders"] == [r] and plan["self_pos"] == 0 and plan["weights"][0] == np.float32(1.0)
+            if tau > 0 and (k < tau or (k - tau) % period):
+                assert plan["senders"] == []                 # nothing was sent tau steps ago
+        x, w = new_x, new_w
+    rng = np.random.default_rng(5)
+    x0 = rng.standard_normal((n, d))
+    st = osgp.sgp_run(x0, K, P_of_k, lambda k, z: grads[k], lr, tau=tau, send_period=period)
+    assert np.allclose(x, st.x, rtol=1e-6, atol=1e-7) and np.allclose(w, st.w, rtol=1e-6, atol=1e-7)   # fp32 plan weights
+
+
 def _random_custom_schedule(n, steps, seed):
     """Random column-stochastic schedule with NON-uniform fp32 weights (every column sums to 1 in fp32 exactly
     enough for the compiler's check): per sender a random out-set incl. self and Dirichlet-like weights."""
