@@ -339,9 +339,10 @@ def test_param_deviation_matches_oracle(binding, inputs):
         assert np.all(h.param_deviation(A) <= 1e-5)                   # consensus: zero deviation
 
 
-@pytest.mark.parametrize("variant", [1, 3])
-def test_steps_can_be_captured_in_a_cuda_graph(binding, inputs, variant):
-    """One schedule period captured once and replayed: same bits as eager launches (launch-bound small cases)."""
+@pytest.mark.parametrize("variant,lockstep", [(1, 0), (3, 0), (1, 2), (1, 4)])
+def test_steps_can_be_captured_in_a_cuda_graph(binding, inputs, variant, lockstep):
+    """One schedule period captured once and replayed: same bits as eager launches (launch-bound small cases); the
+    cluster launches of the lockstep mode are captured like any other."""
     w = inputs.sweep_workload(16, 10_000)
     n, d = w.n, w.d
     period = 10
@@ -359,6 +360,7 @@ def test_steps_can_be_captured_in_a_cuda_graph(binding, inputs, variant):
     X2, W2, M2, Z2 = fresh()
     with binding.Sgp(n, d, graph_desc(w, binding)) as h:
         h.set_option("variant", variant)
+        h.set_option("lockstep", lockstep)
         h.step(X2, W2, M2, G[0], Z2, 0, w.lr, w.momentum, 0.0, True)       # warm-up outside capture (sets attributes)
         torch.cuda.synchronize()
         X2, W2, M2, Z2 = fresh()
@@ -372,6 +374,7 @@ def test_steps_can_be_captured_in_a_cuda_graph(binding, inputs, variant):
         graph.replay()
         torch.cuda.synchronize()
         assert h.device_status() == 0
+        assert h.get_option("last_lockstep") == lockstep
     for a, b in ((X, X2), (W, W2), (M, M2), (Z, Z2)):
         assert torch.equal(a, b)
 
