@@ -13,7 +13,8 @@
  * (Sec. 2 "Approximate distributed averaging"; supplementary "Modeling message delays").
  *
  * Layout advice: make ld a multiple of 256 floats so that every row starts on a 1 KB boundary; the step then
- * runs at ~0.98 of the device's copy bandwidth instead of ~0.88 with the dense pitch ld = d.
+ * runs at ~0.98 of the device's copy bandwidth instead of ~0.91 with a dense pitch ld = d whose rows start off
+ * the 128-byte grid.
  *
  * Every function returns an int status (SGP_OK = 0, negative = error), never throws, aborts or prints.
  * Kernels are enqueued on the caller's stream (a cudaStream_t passed as void*) and the calls return
@@ -275,7 +276,7 @@ int sgp_param_deviation(sgp_handle *h, const float *d_A, double *h_dev, void *st
  *   "tile_cols"    columns per tile (multiple of 4; 0 = automatic)
  *   "ctas_per_sm"  persistent CTAs per SM (0 = automatic)
  *   "stages"       shared-memory stages of the bulk-copy pipeline (0 = automatic, at most 8)
- *   "single_buffer" register-staged kernel: 0 = automatic (n > 128), 1 = one exchange tile and two barriers
+ *   "single_buffer" register-staged kernel: 0 = automatic (from n and the tile width), 1 = one exchange tile and two barriers
  *                  per tile, 2 = two exchange tiles and one barrier
  *   "lockstep"     register-staged kernel: 2 or 4 = launch it as thread-block clusters of that many CTAs that take
  *                  neighbouring tiles and meet at a cluster barrier before each tile (they share no data; it only
