@@ -4,7 +4,7 @@
 //              message slot in this GPU's memory together with w_i                  (Alg. 1 line 5: the "send")
 //     mix      x_i' = sum_j p_ij h_j ,  w_i' = sum_j p_ij w_j ,  z_i = x_i' / w_i'  (Alg. 1 lines 6-8)
 // where the mix reads the in-neighbours' slots straight out of THEIR GPU's memory with plain 128-bit loads over
-// NVLink (peer pointers; no staging copy, no landing buffer, no multicast): the pull and the mix are one kernel.
+// NVLink (peer pointers; no staging copy, no landing buffer, every reader issues its own loads): the pull and the mix are one kernel.
 // With a delay tau >= 1 (Alg. 2) the messages consumed at step k were published at step k - tau, so nothing the
 // kernel reads is still being written and update + pull + mix fuse into ONE kernel per step.
 //

@@ -5,7 +5,7 @@
 // segments are what keeps HBM below its streaming rate.  Here every CTA of the cluster holds a slice of the rows
 // (rows_per_cta = a power of two >= n / cluster size) at FOUR times the tile width, and the gather reads
 // neighbour rows out of the sibling CTAs' shared memory (distributed shared memory, plain ld through
-// map_shared_rank; no multicast, no TMA).  Two cluster barriers per tile: after the half steps are written, and
+// map_shared_rank).  Two cluster barriers per tile: after the half steps are written, and
 // before the tile is overwritten.  Nothing else differs from the register-staged kernel: same local update, same
 // CSR order, same FMA chain, bit-identical results.
 #pragma once

@@ -10,7 +10,7 @@ namespace sgp {
 // segment of X, G (and M, ring) -- into a ring of shared-memory stages with cp.async.bulk, completion
 // counted on an mbarrier per stage; eight consumer warps update, exchange through the stage itself
 // (x^(k+1/2) overwrites the X tile in place), gather-mix and store with 128-bit streaming stores.
-// Loads therefore stay in flight while the consumers compute and store.  No multicast, no cluster.
+// Loads therefore stay in flight while the consumers compute and store.  Every CTA fetches its own tiles; no cluster.
 // Every wait is bounded: on expiry the CTA records a status bit and leaves.
 // ------------------------------------------------------------------------------------------------
 constexpr int kTmaConsumers = 256;
