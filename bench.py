@@ -262,7 +262,8 @@ def run_reference(args, w):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64", "data": "synthetic",
-        "config": workload_config(w, extra={"sample_cols": sample_cols}),
+        "config": workload_config(w, extra={"parallelism": f"replicas x{args.gpus}"}),
+        "sample_cols": sample_cols,
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
                          "blas_threads_for_the_mix": threads},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -716,8 +717,9 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
             "ms_per_step": max_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
-            "config": workload_config(w, extra={"gradient_pool": pool, "parallelism": f"replicas x{world}",
-                                                "row_pitch_floats": ld, **launch}),
+            # the same keys and values as the reference arm's line; how this arm laid the workload out is in "launch"
+            "config": workload_config(w, extra={"parallelism": f"replicas x{world}"}),
+            "launch": {"gradient_pool": pool, "row_pitch_floats": ld, **launch},
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": gpu_launches,
             "clocks": sampler.summary(),
         }
