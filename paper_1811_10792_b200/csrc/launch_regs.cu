@@ -213,7 +213,13 @@ int launch_regs(const DeviceInfo &dev, StepParams p, const ConstTable *ct, int u
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
     e = cudaLaunchKernelEx(&cfg, kern, p, ct != nullptr ? *ct : kEmptyTable);
-  } else {
+    if (e != cudaSuccess) {
+      // a cluster launch that the device refuses is only a lost optimisation: launch independent CTAs instead
+      (void)cudaGetLastError();
+      p.lockstep = 0;
+    }
+  }
+  if (!p.lockstep) {
     kern<<<static_cast<unsigned>(grid), kThreads, smem, stream>>>(p, ct != nullptr ? *ct : kEmptyTable);
     e = cudaGetLastError();
   }
