@@ -46,14 +46,18 @@ inline int update_kind(float momentum, int nesterov) {
 
 // Grid of a streaming rank kernel: exactly the CTAs that are resident at once (one wave, grid-stride inside), so
 // that no partial second wave is left at the end of a launch that lasts only ~100 us.
+// `cap` bounds the CTAs per SM: the fused overlap kernel (four to five loads and as many stores per vector) is
+// fastest with four (0.911 of the copy bandwidth against 0.896 with the five to six the occupancy query allows and
+// 0.82 with three); the lighter update and mix kernels want every CTA they can get (0.92 with eight, 0.83 with four).
 template <typename Kernel>
-unsigned stream_grid(const sgp_rank *r, bool vec, Kernel kern) {
+unsigned stream_grid(const sgp_rank *r, bool vec, Kernel kern, int cap = 64) {
   const int64_t work = vec ? std::max<int64_t>(1, r->d >> 2) : r->d;
   int per_sm = 0;
   if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, sgp::kRankThreads, 0) != cudaSuccess || per_sm < 1) {
     (void)cudaGetLastError();
     per_sm = 4;
   }
+  per_sm = std::min(per_sm, cap);
   return static_cast<unsigned>(std::max<int64_t>(1, std::min<int64_t>((work + sgp::kRankThreads - 1) / sgp::kRankThreads,
                                                                       static_cast<int64_t>(r->sm_count) * per_sm)));
 }
@@ -182,8 +186,9 @@ int sgp_rank_create(sgp_rank **out, int rank, int world, int64_t d, const sgp_gr
   r->slots = tau + 2;
   r->flags = flags;
   r->d = d;
-  r->w_offset = (d + 31) / 32 * 32;
-  r->slot_floats = r->w_offset + 32;
+  // every slot starts on a 1 KB boundary (the row-pitch lesson of the stacked kernels); the weight sits in the pad
+  r->w_offset = (d + 255) / 256 * 256;
+  r->slot_floats = r->w_offset + 256;
   r->sched = sched;
   r->peer_block.assign(static_cast<size_t>(world), nullptr);
   auto fail = [&](int code) {
@@ -309,18 +314,20 @@ int rank_overlap(sgp_rank *r, float *d_x, float *d_w, float *d_m, float *d_v, co
   const bool vec = aligned16(d_x) && aligned16(d_g) && (d_m == nullptr || aligned16(d_m)) && (d_v == nullptr || aligned16(d_v)) &&
                    (d_z == nullptr || aligned16(d_z));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+#define SGP_LAUNCH_CAPPED(KERNEL, ...) KERNEL<<<stream_grid(r, vec, KERNEL, 4), sgp::kRankThreads, 0, st>>>(__VA_ARGS__)
 #define SGP_LAUNCH_OVERLAP(VEC, HZ)                                                                          \
   switch (upd) {                                                                                             \
-    case sgp::kUpdSgd: SGP_LAUNCH_ONE((sgp::sgp_rank_overlap_kernel<VEC, sgp::kUpdSgd, HZ>), p, s); break;    \
-    case sgp::kUpdHeavyBall: SGP_LAUNCH_ONE((sgp::sgp_rank_overlap_kernel<VEC, sgp::kUpdHeavyBall, HZ>), p, s); break; \
-    case sgp::kUpdNesterov: SGP_LAUNCH_ONE((sgp::sgp_rank_overlap_kernel<VEC, sgp::kUpdNesterov, HZ>), p, s); break; \
-    default: SGP_LAUNCH_ONE((sgp::sgp_rank_overlap_kernel<VEC, sgp::kUpdAdam, HZ>), p, s);                    \
+    case sgp::kUpdSgd: SGP_LAUNCH_CAPPED((sgp::sgp_rank_overlap_kernel<VEC, sgp::kUpdSgd, HZ>), p, s); break;    \
+    case sgp::kUpdHeavyBall: SGP_LAUNCH_CAPPED((sgp::sgp_rank_overlap_kernel<VEC, sgp::kUpdHeavyBall, HZ>), p, s); break; \
+    case sgp::kUpdNesterov: SGP_LAUNCH_CAPPED((sgp::sgp_rank_overlap_kernel<VEC, sgp::kUpdNesterov, HZ>), p, s); break; \
+    default: SGP_LAUNCH_CAPPED((sgp::sgp_rank_overlap_kernel<VEC, sgp::kUpdAdam, HZ>), p, s);                    \
   }
   if (vec) {
     if (d_z) { SGP_LAUNCH_OVERLAP(4, true) } else { SGP_LAUNCH_OVERLAP(4, false) }
   } else {
     if (d_z) { SGP_LAUNCH_OVERLAP(1, true) } else { SGP_LAUNCH_OVERLAP(1, false) }
   }
+#undef SGP_LAUNCH_CAPPED
 #undef SGP_LAUNCH_OVERLAP
   SGP_RANK_TRY(r, cudaGetLastError());
   return SGP_OK;
