@@ -244,10 +244,25 @@ def _ptr(t):
     return None if t is None else C.c_void_p(t.data_ptr())
 
 
+_torch = None
+
+
+def _get_torch():
+    global _torch
+    if _torch is None:
+        import torch
+        _torch = torch
+    return _torch
+
+
 def _stream_ptr(stream):
-    import torch
-    s = torch.cuda.current_stream() if stream is None else stream
-    return C.c_void_p(s.cuda_stream)
+    if stream is not None:
+        return C.c_void_p(stream.cuda_stream)
+    torch = _get_torch()
+    raw = getattr(torch._C, "_cuda_getCurrentRawStream", None)      # the current stream's handle without a Stream object
+    if raw is not None:
+        return C.c_void_p(raw(torch.cuda.current_device()))
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
 
 
 class Sgp:
@@ -283,15 +298,15 @@ class Sgp:
         return _ScheduleView(p, self.n)
 
     def _check_mat(self, t, name, allow_none=False):
-        import torch
         if t is None:
             if allow_none:
                 return
             raise ValueError(f"{name} is required")
-        if t.dtype != torch.float32 or not t.is_cuda:
+        if t.dtype != _get_torch().float32 or not t.is_cuda:
             raise ValueError(f"{name} must be a float32 CUDA tensor")
-        if t.dim() != 2 or t.shape[0] != self.n or t.shape[1] != self.d or t.stride(1) != 1 or \
-                (self.n > 1 and t.stride(0) != self.ld):
+        shape, stride = t.shape, t.stride()
+        if len(shape) != 2 or shape[0] != self.n or shape[1] != self.d or stride[1] != 1 or \
+                (self.n > 1 and stride[0] != self.ld):
             raise ValueError(f"{name} must be n x d with row pitch ld={self.ld}")
 
     def step(self, X, W, M, G, Z, k: int, lr: float, momentum: float = 0.0, weight_decay: float = 0.0,
