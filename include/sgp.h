@@ -276,6 +276,8 @@ int sgp_param_deviation(sgp_handle *h, const float *d_A, double *h_dev, void *st
  *                  maps, 3 = the same kernel fed by one bulk copy per row segment (no tensor maps), 4 = the
  *                  thread-block-cluster kernel (a cluster of CTAs shares a tile through distributed shared memory)
  *                  -- measured slower than variant 1 at every shape tried, never chosen automatically
+ *                  5 = the peeled kernel that the automatic choice takes for rows off the 16-byte grid (each row is
+ *                  cut at its own 16-byte boundaries; with aligned rows it runs too, a little slower than variant 1)
  *   "cluster"      CTAs per cluster of variant 4: 0 = 2, 1 = do not use clusters, 2 or 4
  *   "tile_cols"    columns per tile (multiple of 4; 0 = automatic)
  *   "ctas_per_sm"  persistent CTAs per SM (0 = automatic)

@@ -11,8 +11,8 @@ CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libsgp.so")
 
 SOURCES = ["regs_inst_v4.cu", "regs_inst_v4_diag.cu", "regs_inst_v1.cu", "regs_inst_v1_diag.cu", "tma_inst.cu",
-           "tma_inst_diag.cu", "sgp_api.cu", "launch_regs.cu", "launch_tma.cu", "launch_cluster.cu", "sgp_static.cu", "sgp_rank.cu", "schedule.cpp"]
-HEADERS = ["step_common.cuh", "step_regs_kernel.cuh", "step_tma_kernel.cuh", "step_cluster_kernel.cuh", "regs_instances.inc",
+           "tma_inst_diag.cu", "sgp_api.cu", "launch_regs.cu", "launch_tma.cu", "launch_cluster.cu", "launch_peel.cu", "sgp_static.cu", "sgp_rank.cu", "schedule.cpp"]
+HEADERS = ["step_common.cuh", "step_regs_kernel.cuh", "step_tma_kernel.cuh", "step_cluster_kernel.cuh", "step_peel_kernel.cuh", "regs_instances.inc",
            "tma_instances.inc", "aux_kernels.cuh", "rank_kernels.cuh", "launch.h", "schedule.h"]
 
 NVCC_FLAGS = [

@@ -63,6 +63,19 @@ struct RegsOptions {
 int launch_regs(const DeviceInfo &dev, StepParams p, const ConstTable *ct, int upd, int vec, bool uniform_rows,
                 const RegsOptions &opt, cudaStream_t stream, LaunchRecord *rec);
 
+struct PeelOptions {
+  int64_t tile_cols = 0;          // 0 = automatic
+  int cps = 0;                    // CTAs per SM, 0 = as many as are resident
+  int single_buffer = 0;          // 0 automatic, 1 one tile, 2 two tiles
+};
+// True when the peeled kernel can take the launch: every array at the same distance (a multiple of 4 bytes) from a
+// 16-byte boundary, no fused diagnostics.
+bool peel_applicable(const StepParams &p);
+// One launch of the peeled kernel (rows that do not start on 16-byte boundaries) over columns [p.col_begin, p.col_end).
+// Returns SGP_ERR_STATE when it is not applicable; the caller then uses the scalar instantiation.
+int launch_peel(const DeviceInfo &dev, StepParams p, const ConstTable *ct, int upd, const PeelOptions &opt, cudaStream_t stream,
+                LaunchRecord *rec);
+
 struct TmaOptions {
   int variant = 3;                // 2 = 2-D tensor maps, 3 = one bulk copy per row segment
   int64_t tile_cols = 256;

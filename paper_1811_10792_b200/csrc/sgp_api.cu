@@ -226,7 +226,7 @@ Plan make_plan(const sgp_handle *h, int arrays, bool has_m, int nnz, bool vec) {
   if (vec && h->opt_diagnostics && has_m && pl.variant >= 2) pl = Plan{1, sgp::regs_tile_cols(h->n, 4 * 1024), 2, 0};
   if (h->opt_variant > 0 && (h->opt_variant == 1) != (pl.variant == 1)) {
     // the caller forces the other kernel family: take that family's defaults
-    if (h->opt_variant == 1 || h->opt_variant == 4) {
+    if (h->opt_variant == 1 || h->opt_variant >= 4) {
       pl = Plan{1, vec ? sgp::regs_tile_cols(h->n, 4 * 1024) : 0, 2, 0};
     } else {
       pl = Plan{static_cast<int>(h->opt_variant), 256, 2, 2};
@@ -340,6 +340,28 @@ int launch_step_range(sgp_handle *h, const StepArgs &a, int64_t c0, int64_t c1, 
   const int64_t vec_end = vec_ok ? c0 + ((c1 - c0) & ~int64_t{3}) : c0;
   const int arrays = 2 + (a.M != nullptr ? 1 : 0) + (a.V != nullptr ? 1 : 0) + (h->tau > 0 ? 1 : 0);
   const int nnz = static_cast<int>(csr_of(h, slot_of(h, a.k)).col.size());
+  // Rows that do not start on 16-byte boundaries (ld not a multiple of 4, or every array offset alike): the peeled
+  // kernel cuts each row at its own boundaries and keeps 128-bit accesses (about twice the scalar instantiation's
+  // speed).  Steps whose rows of P are all alike keep the shared-column-sum path of the scalar instantiation.
+  {
+    const size_t slot = slot_of(h, a.k);
+    const bool shortcut = h->tau == 0 && csr_of(h, slot).uniform_rows;
+    const bool want_peel = h->opt_variant == 5 || (h->opt_variant == 0 && !vec_ok && !shortcut);
+    if (want_peel && !h->opt_diagnostics && c1 - c0 >= 16) {
+      StepParams p{};
+      fill_params(h, a, c0, c1, update_w, &p);
+      sgp::PeelOptions po;
+      po.tile_cols = h->opt_tile_cols;
+      po.cps = static_cast<int>(h->opt_ctas_per_sm);
+      po.single_buffer = static_cast<int>(h->opt_single_buffer);
+      sgp::LaunchRecord rec;
+      const int rc = sgp::launch_peel(h->dev, p, h->const_ok[slot] ? &h->const_tables[slot] : nullptr, a.upd, po, stream, &rec);
+      if (rc != SGP_ERR_STATE) {
+        record_launch(h, rec, rc);
+        return rc;
+      }
+    }
+  }
   if (vec_end > c0) {
     Plan pl = make_plan(h, arrays, a.M != nullptr, nnz, true);
     // short rows (fewer 1 KB tiles than SMs): the register kernel with narrow tiles spreads them better
@@ -916,7 +938,7 @@ int sgp_param_deviation(sgp_handle *h, const float *d_A, double *h_dev, void *st
 int sgp_set_option(sgp_handle *h, const char *key, int64_t value) {
   if (h == nullptr || key == nullptr || value < 0) return SGP_ERR_ARG;
   if (std::strcmp(key, "variant") == 0) {
-    if (value > 4) return SGP_ERR_ARG;
+    if (value > 5) return SGP_ERR_ARG;
     h->opt_variant = value;
   } else if (std::strcmp(key, "cluster") == 0) {
     if (value != 0 && value != 1 && value != 2 && value != 4) return SGP_ERR_ARG;

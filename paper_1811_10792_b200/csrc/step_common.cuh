@@ -69,6 +69,8 @@ struct StepParams {
   int inject_stall;    // TMA kernel, fault-injection for tests: CTA 0 never requests its first tile, so its
                        // consumers' bounded wait runs out and the status word is set (nothing hangs)
   int biased;          // 1: z = x, the push-sum weight is left out of the de-bias (Table 4, biased OSGP)
+  int peel_phase0;     // peeled kernel: floats between the last 16-byte boundary and element (row 0, col_begin)
+  int peel_phase_step; // peeled kernel: ld mod 4, what a row adds to that distance
   int lockstep;        // register kernel: > 0 = launched as clusters of this many CTAs that take neighbouring tiles and
                        // meet at a cluster barrier before each tile (no data is shared between them)
   float lr, momentum, wd;

@@ -533,6 +533,54 @@ def test_every_node_count_launches(binding, inputs, tau, diag):
         assert torch.isfinite(X).all() and torch.isfinite(Z).all(), n
 
 
+# ------------------------------------------------------------------ peeled kernel (rows off the 16-byte grid)
+@pytest.mark.parametrize("n,d,pad,offset,tau,momentum", [
+    (32, 4_101, 0, 0, 0, 0.9), (32, 4_102, 0, 0, 1, 0.9), (32, 4_103, 0, 0, 0, 0.0), (5, 1_029, 1, 0, 2, 0.9),
+    (16, 3_000, 3, 1, 0, 0.9), (16, 3_000, 0, 3, 1, 0.9), (64, 2_049, 0, 2, 0, 0.9), (256, 1_031, 0, 0, 0, 0.9),
+    (130, 777, 2, 1, 3, 0.9), (1, 19, 0, 1, 0, 0.9), (3, 16, 1, 0, 1, 0.0), (8, 70_003, 0, 0, 0, 0.9)])
+def test_peeled_kernel_matches_oracle_and_scalar_instantiation(binding, inputs, n, d, pad, offset, tau, momentum):
+    """Rows that do not start on 16-byte boundaries (ld = d + pad not a multiple of 4 and / or every array offset by the
+    same odd number of floats): the automatic choice is the peeled kernel (last_variant 5), whose results are those of
+    the scalar instantiation bit for bit and within tolerance of the oracle.  Shapes cover every row phase, one-row
+    and many-row tiles, tiles narrower than four columns of slack, the delay ring and plain SGD."""
+    w = dataclasses.replace(inputs.sweep_workload(n, d), tau=tau, momentum=momentum, weight_decay=1e-3, K=5)
+    a = _run_gpu(binding, inputs, w, ld=d + pad, offset=offset)
+    _compare(w, a)
+    b = _run_gpu(binding, inputs, w, ld=d + pad, offset=offset, options={"variant": 1})
+    for name in ("X", "Z", "W") + (("M",) if momentum else ()):
+        assert np.array_equal(a[name], b[name]), name
+    if tau:
+        assert np.array_equal(a["ring"][0], b["ring"][0]) and np.array_equal(a["ring"][1], b["ring"][1])
+
+
+@pytest.mark.parametrize("pad,offset,want", [(1, 0, 5), (0, 1, 5), (0, 0, 1), (4, 4, 1)])
+def test_peeled_kernel_is_the_automatic_choice_off_the_16_byte_grid(binding, inputs, pad, offset, want):
+    w = inputs.sweep_workload(16, 40_000)
+    n, d, ld = w.n, w.d, w.d + pad
+    def alloc():
+        buf = torch.zeros(n * ld + offset + 8, device=DEV)
+        return buf[offset:offset + n * ld].view(n, ld)[:, :d]
+    X, M, Z, G = alloc(), alloc(), alloc(), alloc()
+    W = torch.ones(n, device=DEV)
+    with binding.Sgp(n, d, graph_desc(w, binding), ld=ld) as h:
+        h.step(X, W, M, G, Z, 0, w.lr, w.momentum, 0.0, True)
+        torch.cuda.synchronize()
+        assert h.get_option("last_variant") == want and h.device_status() == 0
+        h.set_option("variant", 5)                      # forced: runs on aligned rows as well
+        h.step(X, W, M, G, Z, 1, w.lr, w.momentum, 0.0, True)
+        torch.cuda.synchronize()
+        assert h.get_option("last_variant") == 5 and h.device_status() == 0
+
+
+def test_peeled_kernel_on_aligned_rows_equals_the_vector_kernel(binding, inputs):
+    w = dataclasses.replace(inputs.sweep_workload(32, 9_004), tau=1, K=6, weight_decay=1e-3)
+    a = _run_gpu(binding, inputs, w, options={"variant": 5})
+    _compare(w, a)
+    b = _run_gpu(binding, inputs, w, options={"variant": 1})
+    for name in ("X", "Z", "M", "W"):
+        assert np.array_equal(a[name], b[name]), name
+
+
 # ------------------------------------------------------------------ lockstep clusters of the register-staged kernel
 @pytest.mark.parametrize("n,d,tau,size,diag", [(32, 1_029, 0, 2, 0), (32, 70_001, 1, 2, 0), (64, 9_003, 0, 4, 0), (5, 2_000, 2, 4, 0),
                                                (130, 2_052, 0, 4, 0), (2, 260, 0, 2, 0), (48, 40_000, 1, 2, 1), (8, 300_001, 0, 4, 1)])
