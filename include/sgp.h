@@ -157,8 +157,10 @@ int sgp_get_schedule(const sgp_handle *h, const sgp_schedule **s);
  * a sum of a few interleaved partial sums and shared by all receivers.
  * X, W, M are updated in place; G is only read; Z is only written.  All arrays n x ld fp32 device
  * memory except W (n floats).  Arrays must not overlap.  If every pointer is 16-byte aligned and
- * ld is a multiple of 4 the 128-bit path runs, otherwise a scalar path with the same results at about 0.4 of the
- * copy bandwidth (a dense pitch ld = d with d not a multiple of 4 lands there: pad ld instead).
+ * ld is a multiple of 4 the 128-bit path runs.  Otherwise, if all arrays sit at the same distance from a 16-byte
+ * boundary (a dense pitch ld = d with d not a multiple of 4), a kernel that cuts every row at its own 16-byte
+ * boundaries runs at about 0.7 of the copy bandwidth; anything else takes a scalar path at about 0.4.  Same results
+ * in every case; padding ld is the better answer.
  * k >= 0 selects the schedule slot k mod period and the ring slot k mod tau; for tau > 0 the caller
  * must present k = 0, 1, 2, ... in order.  Asynchronous on `stream`; calls on the same handle must
  * be stream-ordered with respect to each other.
