@@ -221,11 +221,13 @@ def test_ring_export_import_resumes_bit_exactly(binding, inputs):
         assert ei.value.code == binding.SGP_ERR_STATE
 
 
-def test_step_host_matches_device_step(binding, inputs):
-    """Host-buffer entry point (chunked copy/compute pipeline) == device entry point, bit for bit."""
+@pytest.mark.parametrize("d", [50_004, 50_005])
+def test_step_host_matches_device_step(binding, inputs, d):
+    """Host-buffer entry point (chunked copy/compute pipeline) == device entry point, bit for bit; d = 50,005 with the
+    dense pitch puts the rows off the 16-byte grid, so every chunk runs the peeled kernel from its own first column."""
     import dataclasses
     for tau in (0, 1):
-        w = dataclasses.replace(inputs.sweep_workload(16, 50_004), tau=tau, K=4)
+        w = dataclasses.replace(inputs.sweep_workload(16, d), tau=tau, K=4)
         n, d = w.n, w.d
         X = inputs.initial_x(w, device=DEV).contiguous(); W = torch.ones(n, device=DEV)
         M = torch.zeros((n, d), device=DEV); Z = torch.empty((n, d), device=DEV); G = torch.empty((n, d), device=DEV)
