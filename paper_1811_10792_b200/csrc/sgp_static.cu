@@ -179,6 +179,20 @@ extern "C" int sgp_step_static(int n, int64_t d, int64_t ld, const int32_t *h_ro
     const int r = launch(s, dev, p, 4, 0, vec_end, vec_end == d, upd, uniform_rows, st);
     if (r != SGP_OK) return r;
   }
+  if (vec_end == 0 && !uniform_rows && d >= 16) {
+    // rows off the 16-byte grid: the peeled kernel, as on the handle path
+    sgp::StepParams q = p;
+    q.col_begin = 0;
+    q.col_end = d;
+    q.update_w = 1;
+    sgp::DeviceInfo di;
+    di.device = dev;
+    di.sm_count = s.sm_count;
+    di.smem_optin = s.smem_optin;
+    sgp::LaunchRecord rec;
+    const int r = sgp::launch_peel(di, q, nullptr, upd, sgp::PeelOptions{}, st, &rec);
+    if (r != SGP_ERR_STATE) return r;
+  }
   if (vec_end < d) return launch(s, dev, p, 1, vec_end, d, true, upd, uniform_rows, st);
   return SGP_OK;
 }
