@@ -157,8 +157,11 @@ int launch_regs(const DeviceInfo &dev, StepParams p, const ConstTable *ct, int u
   // Order of instructions inside a phase (momentum updates without a ring): every gather of a batch before its
   // stores wins where the tile is made of full four-item batches and row segments are at least 512 bytes (n = 4..96:
   // +1 to +1.7 % of the copy bandwidth) and loses elsewhere (n = 24, three-item batches: 0.935 against 0.974; ragged
-  // last batch, n = 104, 112: 0.89 against 0.92-0.93; 256-byte segments, n = 128, 256: 0.91 against 0.93).
-  const bool gather_first = (static_cast<int64_t>(n) * tv) % (4 * kThreads) == 0 && tile_cols * 4 >= 512;
+  // last batch, n = 104, 112: 0.89 against 0.92-0.93; 256-byte segments, n = 128, 256: 0.91 against 0.93).  It also
+  // costs a launch about 4 us more than it returns below ~0.4 ms of work (n = 64, d = 1e6: 0.267 ms against 0.259;
+  // n = 16, d = 1e7, 0.6 ms: 0.604 against 0.607), so short launches keep the interleaved order.
+  const bool gather_first = (static_cast<int64_t>(n) * tv) % (4 * kThreads) == 0 && tile_cols * 4 >= 512 &&
+                            static_cast<int64_t>(n) * ncols >= (int64_t{1} << 27);
   RegsKernel kern = regs_kernel(vec, upd, p.Z != nullptr, has_ring, p.diag != nullptr, gather_first);
   KernelInfo ki;
   {
