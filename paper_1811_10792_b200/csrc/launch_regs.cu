@@ -179,6 +179,12 @@ int launch_regs(const DeviceInfo &dev, StepParams p, const ConstTable *ct, int u
     cps = std::max(1, std::min({by_regs, by_smem, 2048 / kThreads}));
   }
   int64_t grid = std::min<int64_t>(ntiles, static_cast<int64_t>(dev.sm_count) * cps);
+  // Short launches: with k = ceil(ntiles / grid) tiles for the busiest CTA, ceil(ntiles / k) CTAs finish at the same
+  // time; the few CTA slots left empty cost less than a last round in which most of the device idles.
+  if (grid > 0 && ntiles > grid && ntiles < 32 * grid) {
+    const int64_t rounds = (ntiles + grid - 1) / grid;
+    grid = (ntiles + rounds - 1) / rounds;
+  }
   static const ConstTable kEmptyTable{};
   // Lockstep clusters (what was measured, of the copy bandwidth): rows that do not start on 128-byte boundaries
   // split every 1 KB block between two tiles, and CTAs that take neighbouring tiles at the same moment get most of
