@@ -95,6 +95,14 @@ def test_resnet50_full_size(binding, inputs, ld_align):
     _run_full(binding, inputs, inputs.WORKLOADS["resnet50"], K=20 if ld_align == 256 else 3, ld_align=ld_align)
 
 
+@pytest.mark.parametrize("name,d", [("resnet50", 25_557_033), ("resnet50_osgp1", 25_557_031), ("transformer", 61_000_001)])
+def test_rows_off_the_16_byte_grid_full_size(binding, inputs, name, d):
+    """Dense pitch with d not a multiple of 4: rows start at every distance from a 16-byte boundary and the step runs
+    the peeled kernel; same sampled windows and whole-array invariants (with the per-column conservation check over
+    all d columns) as the aligned layouts."""
+    _run_full(binding, inputs, dataclasses.replace(inputs.WORKLOADS[name], d=d), K=3, ld_align=1)
+
+
 def test_transformer_full_size(binding, inputs):
     _run_full(binding, inputs, inputs.WORKLOADS["transformer"], K=20)
 
