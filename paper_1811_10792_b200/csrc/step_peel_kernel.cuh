@@ -40,17 +40,18 @@ __device__ __forceinline__ void peel_store(float *ptr, float4 v, unsigned mask) 
   if (mask & 8u) __stcs(ptr + 3, v.w);
 }
 
-// One (row, slot) item of a tile.  Slot k of a row whose first owned element sits `head` floats before its next
-// 16-byte boundary covers the columns rel0 .. rel0 + 3 relative to the tile, rel0 = 4 k - (head ? 4 - head : 0):
-// slot 0 is the partial head (when head > 0), slot tv the partial tail.
+// One (row, slot) item of a tile.  Slot k of a row whose first owned element sits `phase` floats after a 16-byte
+// boundary covers the columns rel0 .. rel0 + 3 relative to the tile, rel0 = 4 k - phase: with phase > 0 slot 0 is the
+// partial head (its first `phase` elements belong to the previous tile) and slot tv the partial tail.
 struct PeelItem {
   int row;
   int rel0;        // first column of the vector relative to the tile's first column (-3 .. T - 1)
   unsigned mask;   // which of its four elements the tile owns
 };
 
-__device__ __forceinline__ int peel_head(const StepParams &p, int row) {
-  return (4 - ((p.peel_phase0 + row * p.peel_phase_step) & 3)) & 3;
+// Floats between the last 16-byte boundary and the row's first element of a tile (the same for every tile and array).
+__device__ __forceinline__ int peel_phase(const StepParams &p, int row) {
+  return (p.peel_phase0 + row * p.peel_phase_step) & 3;
 }
 
 __device__ __forceinline__ PeelItem peel_item(const StepParams &p, int item, int tile_items, int tv, int valid_cols) {
@@ -63,8 +64,7 @@ __device__ __forceinline__ PeelItem peel_item(const StepParams &p, int item, int
     it.row = item - tile_items;          // the extra slot of every row: its partial tail
     k = tv;
   }
-  const int head = peel_head(p, it.row);
-  it.rel0 = 4 * k - (head ? 4 - head : 0);
+  it.rel0 = 4 * k - peel_phase(p, it.row);
   const int lo = max(0, -it.rel0);
   const int hi = min(4, valid_cols - it.rel0);
   it.mask = (it.row < p.n && hi > lo) ? ((0xFu << lo) & (0xFu >> (4 - hi))) : 0u;
@@ -73,8 +73,7 @@ __device__ __forceinline__ PeelItem peel_item(const StepParams &p, int item, int
 
 // Index of column `rel` of `row` in the shared tile: rows are shifted so that rel0 of every slot is a multiple of 4.
 __device__ __forceinline__ int peel_smem_index(const StepParams &p, int row, int pitch, int rel) {
-  const int head = peel_head(p, row);
-  return row * pitch + 4 + ((4 - head) & 3) + rel;
+  return row * pitch + 4 + peel_phase(p, row) + rel;
 }
 
 template <int UPD, bool HAS_Z, bool HAS_RING>
@@ -156,7 +155,7 @@ sgp_step_peel_kernel(const __grid_constant__ StepParams p, const __grid_constant
         const int64_t o = static_cast<int64_t>(me[q].row) * ld + col0 + me[q].rel0;
         // my slot sits 16-byte aligned in my row of the tile; in a sender's row the same columns start `s` floats
         // after a 16-byte boundary, s = difference of the two rows' shifts: two aligned reads and a select
-        const int my_shift = (4 - peel_head(p, me[q].row)) & 3;
+        const int my_shift = peel_phase(p, me[q].row);
         const int my_index = 4 + my_shift + me[q].rel0;                 // a multiple of 4
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f), offd = make_float4(0.f, 0.f, 0.f, 0.f);
         const int e1 = tab.rowptr[me[q].row + 1];
@@ -164,7 +163,7 @@ sgp_step_peel_kernel(const __grid_constant__ StepParams p, const __grid_constant
           const int j = tab.col[e];
           if (!SGP_BOUNDS_OK(p, j >= 0 && j < n)) continue;
           const float pv = tab.val[e];
-          const int delta = ((4 - peel_head(p, j)) & 3) - my_shift;      // -3 .. 3
+          const int delta = peel_phase(p, j) - my_shift;                  // -3 .. 3
           const int s = delta & 3;
           const float4 *src = reinterpret_cast<const float4 *>(H + j * pitch + my_index + (delta < 0 ? -4 : 0));
           const float4 lo4 = src[0];
