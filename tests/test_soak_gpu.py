@@ -70,3 +70,15 @@ def test_three_hundred_checked_steps(binding, inputs, name):
         assert h.get_option("last_variant") == want_variant and h.get_option("last_lockstep") == want_lockstep
         stats = h.check(X, W)
         assert stats["code"] == binding.SGP_OK and stats["nonfinite"] == 0 and abs(stats["sum_w"] - n) < 1e-4 * n
+
+
+@pytest.mark.parametrize("tau,period", [(0, 1), (1, 1), (2, 1), (3, 2)])
+def test_two_hundred_steps_one_node_per_gpu_equal_the_stacked_step(binding, inputs, tau, period):
+    """The message slots of the one-node-per-GPU mode are reused every tau + 2 steps: after 200 steps on a random
+    digraph (weights away from 1) the loopback ranks still hold the stacked step's bits."""
+    from test_rowshard_gpu import _run_both
+    w = dataclasses.replace(inputs.sweep_workload(12, 20_004), tau=tau, weight_decay=1e-4, lr=0.01)
+    _x0, _grads, got, stacked = _run_both(binding, inputs, w, 200, send_period=period)
+    for name in ("X", "Z", "M", "W"):
+        assert torch.equal(got[name], stacked[name]), name
+    assert float(got["W"].max() - got["W"].min()) > 1e-3
