@@ -242,7 +242,8 @@ int sgp_colsum(sgp_handle *h, const float *d_A, int include_ring, double *d_out,
  * bounded wait, else SGP_ERR_INVARIANT if any of the three invariants failed, else SGP_OK.  Synchronises.
  * The weight sum is conserved only to fp32 rounding: weights such as 1/3 make the columns of P sum to 1 within an ulp,
  * and the sum walks away from n by about 4e-5 n per 4000 steps on random digraphs (measured at n = 256), so a run of
- * 1e5 steps and more should read [6] against its own history rather than against the fixed bound.
+ * 1e4 steps and more (n = 256 crosses 1e-4 n after about 10,000 steps) should read [6] against its own history
+ * rather than against the fixed bound; the per-step bracket of "check_steps" compares consecutive sums instead.
  */
 int sgp_check(sgp_handle *h, const float *d_X, const float *d_W, const double *d_colsum_ref, double *h_stats,
               void *stream);
@@ -304,7 +305,9 @@ int sgp_param_deviation(sgp_handle *h, const float *d_A, double *h_dev, void *st
  *                  (sgp_get_diagnostics reads the latest)
  *   "check_steps"  0/1, debug: every step is bracketed by an expected-column-sum pre-pass and a column-sum check
  *                  (sum_i x_i' plus ring against sum_i h_i plus ring, Sec. 2); a drift sets SGP_STATUS_COLUMN_SUM in
- *                  the device status word.  Costs about two extra passes over the arrays and 8 d bytes of device
+ *                  the device status word, and a weight sum (weights in transit included) that differs from the one
+ *                  taken just before the step by more than 1e-5 n sets SGP_STATUS_WEIGHT_SUM (one step keeps the sum
+ *                  to a few roundings).  Costs about two extra passes over the arrays and 8 d bytes of device
  *                  memory, allocated when the option is switched on (SGP_ERR_ALLOC if that fails)
  * Read-only through sgp_get_option: "last_variant", "last_grid", "last_smem", "last_tile_cols", "last_lockstep" describe
  * the most recent step launch of the handle (which kernel ran, CTAs, dynamic shared memory, tile width);

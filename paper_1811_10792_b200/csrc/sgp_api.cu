@@ -428,18 +428,22 @@ int launch_expected(sgp_handle *h, const StepArgs &a, cudaStream_t st) {
     default:
       sgp::sgp_expected_colsum_kernel<sgp::kUpdAdam><<<grid, 256, 0, st>>>(a.X, a.G, a.M, a.V, h->n, h->d, h->ld, us, h->ring_x, ring_rows, h->d_expect);
   }
+  // the weight sum before the step (weights in transit included) lands in d_stats[6] (and the minimum in [7]): the
+  // scan writes at kStatSumW = 2 and kStatMinW = 3 from the pointer it is given
+  sgp::sgp_weight_scan_kernel<<<1, 256, 0, st>>>(a.W, h->n, h->ring_w, h->tau * h->n, h->d_stats + kDevStatsCheck + 4);
   SGP_CUDA_TRY(h, cudaGetLastError());
   return SGP_OK;
 }
 
 // Enqueues the invariant scan of (X, W, ring) against an optional column-sum reference; statistics stay on the
 // device (d_stats) and violations are ORed into the status word.  No synchronisation.
-int enqueue_check(sgp_handle *h, const float *X, const float *W, const double *ref, cudaStream_t st) {
+int enqueue_check(sgp_handle *h, const float *X, const float *W, const double *ref, cudaStream_t st,
+                  const double *sum_before = nullptr) {
   double *stats = h->d_stats + kDevStatsCheck;
   SGP_CUDA_TRY(h, cudaMemsetAsync(stats, 0, sgp::kStatCount * sizeof(double), st));
   sgp::sgp_colsum_kernel<<<column_grid(h), 256, 0, st>>>(X, h->n, h->d, h->ld, h->ring_x, h->tau * h->n, nullptr, ref, stats);
   sgp::sgp_weight_scan_kernel<<<1, 256, 0, st>>>(W, h->n, h->ring_w, h->tau * h->n, stats);
-  sgp::sgp_check_finalize_kernel<<<1, 1, 0, st>>>(stats, h->n, 1, ref != nullptr ? 1 : 0, kColumnDriftTol, h->d_words + 1);
+  sgp::sgp_check_finalize_kernel<<<1, 1, 0, st>>>(stats, h->n, 1, ref != nullptr ? 1 : 0, kColumnDriftTol, h->d_words + 1, sum_before);
   SGP_CUDA_TRY(h, cudaGetLastError());
   return SGP_OK;
 }
@@ -459,7 +463,8 @@ int run_step(sgp_handle *h, const StepArgs &a, cudaStream_t st) {
   }
   const int rc = launch_step_range(h, a, 0, h->d, true, st);
   if (rc != SGP_OK) return rc;
-  if (h->opt_check_steps) return enqueue_check(h, a.X, a.W, h->d_expect, st);
+  // the bracket compares the weight sum with the one taken before the step (d_stats[6]), not with n
+  if (h->opt_check_steps) return enqueue_check(h, a.X, a.W, h->d_expect, st, h->d_stats + kDevStatsCheck + 6);
   return SGP_OK;
 }
 

@@ -49,6 +49,22 @@ for n, variant in ((8, 1), (8, 3), (128, 1)):                       # table in t
         torch.cuda.synchronize()                                    # no fault: the access was skipped
         assert h.device_status() & binding.SGP_STATUS_BOUNDS, (n, variant)
         assert torch.isfinite(X).all().item()
+# the skipped entry is a lost message: with the per-step bracket on, the step's weight sum and column sums no longer
+# match what they were before the step, and both conservation bits are raised (Sec. 2, 1^T P = 1^T)
+n = 8
+w = inputs.sweep_workload(n, 40_000)
+X = inputs.initial_x(w, device="cuda:0").contiguous()
+W = torch.ones(n, device="cuda:0"); M = torch.zeros_like(X); Z = torch.empty_like(X)
+G = inputs.gradient(w, 0, torch.empty_like(X))
+with binding.Sgp(n, w.d, binding.graph_desc(w)) as h:
+    h.set_option("check_steps", 1)
+    for k in range(3):
+        h.step(X, W, M, G, Z, k, w.lr, w.momentum, 0.0, True)
+    assert h.device_status() == 0
+    h.set_option("poke_table", n + 1000)
+    h.step(X, W, M, G, Z, 10, w.lr, w.momentum, 0.0, True)
+    st = h.device_status()
+    assert st & binding.SGP_STATUS_WEIGHT_SUM and st & binding.SGP_STATUS_COLUMN_SUM, st
 print("poke ok")
 """
 
