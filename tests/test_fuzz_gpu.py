@@ -1,6 +1,8 @@
 """Seeded random configurations of the fused step against the float64 oracle: node count, parameter count, row pitch
 and pointer offset, delay, optimiser flavour, graph kind, kernel family, lockstep clusters and diagnostics are drawn
 together, so that combinations no hand-written case lists get exercised (Alg. 1 lines 4-8, Alg. 2, Alg. 3)."""
+import os
+
 import numpy as np
 import pytest
 
@@ -43,8 +45,12 @@ def _draw(case: int):
         diag=bool(rng.rand() < 0.25), opts=opts, seed=int(rng.randint(1, 1 << 30)))
 
 
+# SGP_FUZZ_CASES in the environment widens the three sweeps for a longer run by hand (the draws are seeded by case number)
+_EXTRA = max(1, int(os.environ.get("SGP_FUZZ_CASES", "0")) // 256)
+
+
 @pytest.mark.gpu
-@pytest.mark.parametrize("case", range(256))
+@pytest.mark.parametrize("case", range(256 * _EXTRA))
 def test_random_configuration_matches_oracle(binding, inputs, case):
     c = _draw(case)
     kind, peers = ("exp", 2) if c["graph"] == "exp2" else (c["graph"], 1)
@@ -83,17 +89,47 @@ def _draw_adam(case: int):
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("case", range(64))
+@pytest.mark.parametrize("case", range(64 * _EXTRA))
 def test_random_adam_configuration_matches_oracle(binding, inputs, case):
     """The same for the Adam-preconditioned step (Sec. 6.2 / App. C.1)."""
-    from test_adam_gpu import _compare as adam_compare, _run as adam_run
+    from test_adam_gpu import _run as adam_run
     c = _draw_adam(case)
     kind, peers = ("exp", 2) if c["graph"] == "exp2" else (c["graph"], 1)
     w = inputs.Workload(f"fuzz_adam{case}", n=c["n"], d=c["d"], K=c["K"], graph=kind, peers=peers, max_outdeg=4,
                         num_steps=5, tau=c["tau"], seed=c["seed"], optimizer="adam")
     out = adam_run(binding, inputs, w, options=c["opts"], ld=c["d"] + c["pad"], offset=c["offset"], wd=c["wd"],
                    write_z=c["write_z"])
-    adam_compare(w, out, wd=c["wd"], write_z=c["write_z"])
+    _adam_compare_conditioned(w, out, wd=c["wd"], write_z=c["write_z"])
+
+
+def _adam_compare_conditioned(w, out, wd, write_z, lr=1e-2):
+    """The Adam step divides by sqrt(v) + eps: where the effective gradient g + wd x all but cancels, the ratio is close
+    to sign(g~) and ANY two precisions disagree there by up to 2 lr (about one element in a million with these inputs).
+    Such elements are found from the oracle alone -- the same run with every gradient scaled by 1 + 2^-22, four fp32
+    roundings -- and are held to a bound of 4 K lr instead of the relative tolerance; at most one element in a thousand
+    may be of that kind.  Everything else meets the usual gate."""
+    from oracle import sgp as osgp
+    from test_adam_gpu import BETAS, EPS
+    from parity_util import REL_TOL
+
+    def run(scale):
+        return osgp.sgp_run(out["x0"].astype(np.float64), w.K, oracle_P_of_k(w),
+                            lambda k, z: out["grads"][k].astype(np.float64) * scale, lr, weight_decay=wd, tau=w.tau,
+                            adam=(BETAS[0], BETAS[1], EPS))
+    st, st_eps = run(1.0), run(1.0 + 2.0 ** -22)
+    names = [("X", out["X"], st.x, st_eps.x), ("M1", out["M1"], st.u, st_eps.u), ("M2", out["M2"], st.v, st_eps.v)]
+    if write_z:
+        names.append(("Z", out["Z"], st.z, st_eps.z))
+    for name, got, want, want_eps in names:
+        got = got.astype(np.float64)
+        floor = np.maximum(np.abs(want), np.sqrt(np.mean(want * want)))
+        ill = np.abs(want_eps - want) > 0.5 * REL_TOL * floor
+        assert ill.mean() <= 1e-3, (name, float(ill.mean()))
+        diff = np.abs(got - want)
+        assert np.all(diff[ill] <= 4 * w.K * lr * np.maximum(1.0, np.abs(want[ill]))), name
+        if (~ill).any():
+            assert (diff[~ill] / floor[~ill]).max() <= REL_TOL, (name, float((diff[~ill] / floor[~ill]).max()))
+    assert_close("W", out["W"], st.w)
 
 
 def _draw_rank(case: int):
@@ -111,7 +147,7 @@ def _draw_rank(case: int):
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("case", range(64))
+@pytest.mark.parametrize("case", range(64 * _EXTRA))
 def test_random_one_node_per_gpu_configuration_equals_stacked_step(binding, inputs, case):
     """The split kernels (update / pull + mix, fused overlap step) in loopback give the stacked step's bits
     (App. C setting, Alg. 1 lines 4-8, Alg. 2), whatever the shape, delay, graph and alignment."""
