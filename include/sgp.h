@@ -403,7 +403,9 @@ int sgp_rank_create(sgp_rank **out, int rank, int world, int64_t d, const sgp_gr
 int sgp_rank_destroy(sgp_rank *r);
 int sgp_rank_get_schedule(const sgp_rank *r, const sgp_schedule **s);
 /* The rank's message slots: one device allocation of `bytes` bytes.  Other ranks need its address in THEIR
- * process: the same pointer inside one process, or sgp_ipc_export here + sgp_ipc_open there. */
+ * process: the same pointer inside one process, or sgp_ipc_export here + sgp_ipc_open there.  The block is plain
+ * device memory holding every message still in transit: a checkpoint copies its `bytes` out (with x, u, w) and a
+ * restart copies them back into the block of a rank created with the same arguments before its next step. */
 int sgp_rank_message_block(sgp_rank *r, void **d_block, size_t *bytes);
 /* d_peer_blocks[j] (HOST array of `world` device pointers valid in this process; entry [rank] is ignored, entries
  * of ranks this node never receives from may be NULL): where rank j's message block is mapped. */

@@ -279,3 +279,50 @@ def test_loopback_adam_matches_oracle_and_stacked_step(binding, inputs, n, d, ta
     assert_close("W", got["W"].cpu().numpy(), st.w)
     for name, ref in (("X", X), ("Z", Z), ("M1", M1), ("M2", M2), ("W", W)):
         assert torch.equal(got[name], ref), name
+
+
+def test_messages_in_transit_survive_a_checkpoint_of_the_message_block(binding, inputs):
+    """One node per GPU with tau = 2: the message block of a rank is plain device memory, so copying its bytes out and
+    back (with x, u and w) into a freshly created rank resumes the run bit for bit -- the counterpart of
+    sgp_ring_export / sgp_ring_import for this mode."""
+    try:
+        from cuda.bindings import runtime as cudart
+    except ImportError:
+        from cuda import cudart
+    from paper_1811_10792_b200 import rowshard
+    w = dataclasses.replace(inputs.sweep_workload(8, 3_000), tau=2, weight_decay=1e-3)
+    n, d, K1, K2 = w.n, w.d, 5, 9
+    G = torch.empty((n, d), device=DEV)
+    def fresh_rows():
+        X = inputs.initial_x(w, device=DEV).contiguous()
+        return ([X[r].clone() for r in range(n)], [torch.ones(1, device=DEV) for _ in range(n)],
+                [torch.zeros(d, device=DEV) for _ in range(n)], [torch.empty(d, device=DEV) for _ in range(n)])
+    def run(grp, xs, ws, ms, zs, k0, k1):
+        for k in range(k0, k1):
+            inputs.gradient(w, k, G)
+            gs = [G[r].clone() for r in range(n)]
+            grp.step(xs, ws, ms, gs, zs, k, w.lr, w.momentum, w.weight_decay, True)
+        torch.cuda.synchronize()
+    xs, ws, ms, zs = fresh_rows()
+    with rowshard.LoopbackGroup(n, d, graph_desc(w, binding), tau=w.tau) as grp:
+        run(grp, xs, ws, ms, zs, 0, K1)
+        saved = []
+        for rk in grp.ranks:
+            ptr, size = rk.message_block()
+            buf = torch.empty(size, dtype=torch.uint8, device=DEV)
+            err, = cudart.cudaMemcpy(buf.data_ptr(), ptr, size, cudart.cudaMemcpyKind.cudaMemcpyDeviceToDevice)
+            assert int(err) == 0
+            saved.append(buf)
+        state = ([t.clone() for t in xs], [t.clone() for t in ws], [t.clone() for t in ms])
+        run(grp, xs, ws, ms, zs, K1, K2)
+    xs2, ws2, ms2 = state
+    zs2 = [torch.empty(d, device=DEV) for _ in range(n)]
+    with rowshard.LoopbackGroup(n, d, graph_desc(w, binding), tau=w.tau) as grp2:
+        for rk, buf in zip(grp2.ranks, saved):
+            ptr, size = rk.message_block()
+            assert size == buf.numel()
+            err, = cudart.cudaMemcpy(ptr, buf.data_ptr(), size, cudart.cudaMemcpyKind.cudaMemcpyDeviceToDevice)
+            assert int(err) == 0
+        run(grp2, xs2, ws2, ms2, zs2, K1, K2)
+    for a, b in zip(xs + ws + ms + zs, xs2 + ws2 + ms2 + zs2):
+        assert torch.equal(a, b)
